@@ -1,0 +1,412 @@
+#!/usr/bin/env python
+"""Benchmark of the IKBO hot path on B200.
+
+One step = one pass of the retrieval-MLP workload (configuration 2: R = 256 requests x 512
+candidates, 768 -> 1024 -> 1024 -> 256, first layer split 512 | 256 between request and candidate
+features): segment plan, request half, candidate half with the in-kernel broadcast, and the two
+plain layers.  `value` is candidates scored per second over all ranks with inputs resident in HBM;
+`e2e` is the same step from pinned host buffers (inputs copied in, scores copied out every step).
+Extra keys report each layer against its own roofline, and the attention (configuration 3) and
+interaction (configuration 4) kernels on their own workloads.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl rocs|reference]
+
+`--impl reference` times the fp64 CPU oracle on a bounded sample of the same workload.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+from paper_2607_27744_b200 import workloads as wl  # noqa: E402
+
+METRIC = "candidates scored/sec per IKBO layer (bf16, 1 B200) and % of roofline"
+UNIT = "candidates/s"
+WORKLOAD = "config 2: retrieval MLP bf16, R=256 x 512 candidates (N=131072), 768->1024->1024->256, layer 1 split 512|256"
+N_SETS = 4  # rotating input/output sets: 4 x (67 MB in + 600 MB activations) >> 126 MB L2
+
+
+def measured_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        p = json.load(open(path))
+        return dict(hbm_gbs=p["hbm_gbs"], tflops_burst=p["bf16_tflops"],
+                    tflops_sustained=p.get("bf16_tflops_sustained", p["bf16_tflops"]), source="measured")
+    return dict(hbm_gbs=6650.0, tflops_burst=1590.0, tflops_sustained=1400.0, source="fallback")
+
+
+class ClockSampler:
+    """Samples SM clocks and throttle reasons with nvidia-smi while the timed region runs."""
+    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+              "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.rows, self.proc, self.index = [], None, index
+
+    def __enter__(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", f"--id={self.index}", f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits",
+                 "-lms", "100"], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.thread = threading.Thread(target=self._read, daemon=True)
+            self.thread.start()
+        except OSError:
+            self.proc = None
+        return self
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.rows.append([c.strip() for c in line.split(",")])
+
+    def __exit__(self, *exc):
+        if self.proc:
+            self.proc.terminate()
+            try:
+                self.proc.wait(timeout=5)
+            except subprocess.TimeoutExpired:
+                self.proc.kill()
+            self.thread.join(timeout=5)
+
+    def summary(self):
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for r in self.rows:
+            try:
+                sm.append(float(r[0]))
+                mx.append(float(r[1]))
+            except (ValueError, IndexError):
+                continue
+            for name, v in zip(names, r[3:7]):
+                if v.lower().startswith("active"):
+                    reasons.add(name)
+        if not sm:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        return {"sm_mhz": float(np.median(sm)), "sm_max_mhz": max(mx), "reasons": sorted(reasons),
+                "samples": len(sm)}
+
+
+# --------------------------------------------------------------------------------------------
+# reference arm / cpu baseline: the oracle on a bounded sample
+# --------------------------------------------------------------------------------------------
+def oracle_mlp_rate(n_sample: int, data=None):
+    """Times the oracle's three-layer MLP on `n_sample` candidates of configuration 2.
+    Returns (candidates per second, threads used, seconds)."""
+    from oracle import rocs_ref as ref
+    cfg = wl.CONFIGS[2]
+    if data is None:
+        data = host_inputs(cfg)
+    co, lin, ws = data["co"], data["lin"], data["ws"]
+    N = int(co[-1])
+    sample = np.unique(np.linspace(0, N - 1, n_sample).astype(np.int64))
+    t0 = time.perf_counter()
+    h = ref.ikbo_linear(co, lin["XR"], lin["XC"], lin["W"], relu=True, sample=sample)
+    one = wl.offsets_from_counts([h.shape[0]])
+    h = ref.ikbo_linear(one, None, h, wl.to_f64(ws[0]), relu=True)
+    ref.ikbo_linear(one, None, h, wl.to_f64(ws[1]))
+    dt = time.perf_counter() - t0
+    return sample.size / dt, ref.num_threads(), dt
+
+
+def host_inputs(cfg):
+    co = wl.cand_offsets(cfg)
+    return dict(co=co, lin=wl.linear_inputs(cfg, co), ws=wl.mlp_weights(cfg))
+
+
+def sized_oracle_run(data, target_s: float = 12.0):
+    rate, threads, dt = oracle_mlp_rate(64, data)
+    n = int(max(64, min(int(data["co"][-1]), rate * target_s)))
+    rate, threads, dt = oracle_mlp_rate(n, data)
+    return rate, threads, dt, n
+
+
+def run_reference(args):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    data = host_inputs(wl.CONFIGS[2])
+    probe_rate, threads, _ = oracle_mlp_rate(64, data)
+    budget_s = min(8.0, 120.0 / max(1, args.steps + args.warmup))   # whole run within a few minutes
+    per_step = int(max(8, min(4096, probe_rate * budget_s)))
+    for _ in range(args.warmup):
+        oracle_mlp_rate(per_step, data)
+    t0 = time.perf_counter()
+    done = 0
+    for _ in range(args.steps):
+        oracle_mlp_rate(per_step, data)
+        done += per_step
+    dt = time.perf_counter() - t0
+    value = done / dt
+    print(json.dumps({
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": dt / args.steps * 1e3,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": WORKLOAD, "sample_per_step": per_step},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": threads, "kind": "oracle",
+                         "sample": f"{per_step} evenly spaced candidates of the workload per step, all three layers"},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }))
+
+
+# --------------------------------------------------------------------------------------------
+# CUDA arm
+# --------------------------------------------------------------------------------------------
+def run_rocs(args):
+    import torch
+    from paper_2607_27744_b200 import binding as rocs
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    torch.cuda.set_device(local)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    rocs.lib()  # fail loudly if the CUDA library is missing
+    peaks = measured_peaks()
+    cfg = wl.CONFIGS[2]
+    data = host_inputs(cfg)
+    co = data["co"]
+    N = int(co[-1])
+
+    def dev(a):
+        t = torch.from_numpy(np.ascontiguousarray(a))
+        return (t.view(torch.bfloat16) if a.dtype == np.uint16 else t).cuda()
+
+    def pinned(a):
+        t = torch.from_numpy(np.ascontiguousarray(a))
+        return (t.view(torch.bfloat16) if a.dtype == np.uint16 else t).pin_memory()
+
+    # Requests are independent units (Eq. 1 / Eq. 11): every rank scores its own batch of the same
+    # shape, no collective on the data path (weak scaling).
+    W1 = dev(data["lin"]["W"])
+    W2, W3 = (dev(w) for w in data["ws"])
+    W1_cr, W1_cc = W1[:, :cfg.d_req], W1[:, cfg.d_req:]
+    co_dev = dev(co)
+    XR_sets = [dev(data["lin"]["XR"]) for _ in range(N_SETS)]
+    XC_sets = [dev(data["lin"]["XC"]) for _ in range(N_SETS)]
+    h1 = [torch.empty((N, 1024), dtype=torch.bfloat16, device="cuda") for _ in range(N_SETS)]
+    h2 = [torch.empty((N, 1024), dtype=torch.bfloat16, device="cuda") for _ in range(N_SETS)]
+    y = [torch.empty((N, 256), dtype=torch.bfloat16, device="cuda") for _ in range(N_SETS)]
+    ws_bytes = 256 * 1024 * 4
+    workspace = torch.empty(ws_bytes, dtype=torch.uint8, device="cuda")
+    launches_per_step = 5  # fill_row2req, request half, candidate half, layer 2, layer 3
+
+    def step(i, XR=None, XC=None, co_d=None):
+        s = i % N_SETS
+        plan = rocs.plan_create(co_dev if co_d is None else co_d, co)
+        rocs.ikbo_linear(plan, XR_sets[s] if XR is None else XR, XC_sets[s] if XC is None else XC, W1_cr, W1_cc,
+                         relu=True, out=h1[s], workspace=workspace)
+        rocs.linear(h1[s], W2, relu=True, out=h2[s])
+        rocs.linear(h2[s], W3, out=y[s])
+        plan.close()
+        return y[s]
+
+    def barrier():
+        if dist is not None:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    def ms_estimate(a, b):
+        torch.cuda.synchronize()
+        return a.elapsed_time(b)
+
+    def max_over_ranks(ms):
+        if dist is None:
+            return ms
+        t = torch.tensor([ms], dtype=torch.float64, device="cuda")
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        return float(t.item())
+
+    # ---- device-resident timing -------------------------------------------------------------
+    for i in range(args.warmup):
+        step(i)
+    barrier()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    with ClockSampler(local) as clocks:
+        e0.record()
+        for i in range(args.steps):
+            step(i)
+        e1.record()
+        barrier()
+        if ms_estimate(e0, e1) < 600.0:   # keep the same load running until a few clock samples exist
+            t_end = time.time() + 0.7
+            k = 0
+            while time.time() < t_end:
+                step(k)
+                k += 1
+            torch.cuda.synchronize()
+    ms = max_over_ranks(e0.elapsed_time(e1))
+    rocs.last_device_status()
+    ms_per_step = ms / args.steps
+    value = world * N / (ms_per_step * 1e-3)
+
+    # ---- per-layer timing (CUDA events around each call, same rotating sets) -----------------
+    def time_call(fn, reps=20):
+        for i in range(3):
+            fn(i)
+        torch.cuda.synchronize()
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record()
+        for i in range(reps):
+            fn(i)
+        b.record()
+        torch.cuda.synchronize()
+        return a.elapsed_time(b) / reps * 1e-3
+
+    plan = rocs.plan_create(co_dev, co)
+    t_l1 = time_call(lambda i: rocs.ikbo_linear(plan, XR_sets[i % N_SETS], XC_sets[i % N_SETS], W1_cr, W1_cc, relu=True,
+                                                out=h1[i % N_SETS], workspace=workspace))
+    t_l2 = time_call(lambda i: rocs.linear(h1[i % N_SETS], W2, relu=True, out=h2[i % N_SETS]))
+    t_l3 = time_call(lambda i: rocs.linear(h2[i % N_SETS], W3, out=y[i % N_SETS]))
+    t_plan = time_call(lambda i: rocs.plan_create(co_dev, co).close())
+
+    def layer(name, t, flops, nbytes):
+        t_hbm = nbytes / (peaks["hbm_gbs"] * 1e9)
+        t_tc = flops / (peaks["tflops_burst"] * 1e12)
+        bound = "hbm" if t_hbm >= t_tc else "tensor"
+        ach = nbytes / t / 1e9 if bound == "hbm" else flops / t / 1e12
+        peak = peaks["hbm_gbs"] if bound == "hbm" else peaks["tflops_burst"]
+        return {"layer": name, "us": t * 1e6, "cand_per_s": N / t, "bound": bound, "achieved": ach, "peak": peak,
+                "unit": "GB/s" if bound == "hbm" else "TFLOP/s", "frac": ach / peak,
+                "tflops": flops / t / 1e12, "gbs": nbytes / t / 1e9}
+
+    bf = 2
+    layers = [
+        layer("cfg2.L1 ikbo_linear 512|256->1024 (request half + candidate half)", t_l1,
+              2.0 * N * 256 * 1024 + 2.0 * 256 * 512 * 1024,
+              N * 256 * bf + N * 1024 * bf + 256 * 512 * bf + 1024 * 768 * bf),
+        layer("cfg2.L2 linear 1024->1024", t_l2, 2.0 * N * 1024 * 1024, N * 1024 * bf * 2 + 1024 * 1024 * bf),
+        layer("cfg2.L3 linear 1024->256", t_l3, 2.0 * N * 1024 * 256, N * 1024 * bf + N * 256 * bf + 256 * 1024 * bf),
+    ]
+    dominant = max(layers, key=lambda l: l["us"])
+    roofline = {"kernel": dominant["layer"], "bound": dominant["bound"], "achieved": dominant["achieved"],
+                "peak": dominant["peak"], "unit": dominant["unit"], "frac": dominant["frac"], "traffic": None,
+                "peak_source": peaks["source"] + (" (burst)" if dominant["bound"] == "tensor" else "")}
+
+    # ---- attention and interaction kernels on their own workloads ----------------------------
+    extra = []
+    if not args.skip_extra:
+        extra = bench_other_ops(torch, rocs, peaks, dev, time_call)
+
+    # ---- end to end from pinned host buffers ------------------------------------------------
+    XR_h, XC_h, co_h = pinned(data["lin"]["XR"]), pinned(data["lin"]["XC"]), pinned(co)
+    y_h = torch.empty((N, 256), dtype=torch.bfloat16).pin_memory()
+    XR_d, XC_d, co_d = torch.empty_like(XR_sets[0]), torch.empty_like(XC_sets[0]), torch.empty_like(co_dev)
+
+    def e2e_step(i):
+        XR_d.copy_(XR_h, non_blocking=True)
+        XC_d.copy_(XC_h, non_blocking=True)
+        co_d.copy_(co_h, non_blocking=True)
+        out = step(i, XR_d, XC_d, co_d)
+        y_h.copy_(out, non_blocking=True)
+
+    for i in range(args.warmup):
+        e2e_step(i)
+    barrier()
+    e0.record()
+    for i in range(args.steps):
+        e2e_step(i)
+    e1.record()
+    barrier()
+    e2e_ms = max_over_ranks(e0.elapsed_time(e1)) / args.steps
+    h2d = XR_h.numel() * 2 + XC_h.numel() * 2 + co_h.numel() * 4
+    d2h = y_h.numel() * 2
+
+    if rank != 0:
+        return
+    cpu = None
+    if world == 1 and not args.skip_cpu:
+        rate, threads, dt, n = sized_oracle_run(data)
+        cpu = {"value": rate, "unit": UNIT, "cores": threads, "kind": "oracle",
+               "sample": f"{n} evenly spaced candidates of the workload, all three layers, {dt:.1f} s"}
+    print(json.dumps({
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
+        "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "bf16", "data": "synthetic",
+        "config": {"workload": WORKLOAD, "l2": f"{N_SETS} rotating input/activation sets, larger than L2",
+                   "step": "plan + request half + candidate half (in-kernel broadcast) + 2 plain layers"},
+        "clocks": clocks.summary(),
+        "e2e": {"value": world * N / (e2e_ms * 1e-3), "unit": UNIT, "h2d_bytes_per_step": h2d,
+                "d2h_bytes_per_step": d2h, "ms_per_step": e2e_ms},
+        "gpu_launches": launches_per_step * args.steps,
+        "roofline": roofline,
+        "cpu_baseline": cpu,
+        "layers": layers,
+        "plan_us": t_plan * 1e6,
+        "other_ikbo_layers": extra,
+    }))
+
+
+def bench_other_ops(torch, rocs, peaks, dev, time_call):
+    """Attention on configuration 3 and interaction on configuration 4, one layer each."""
+    out = []
+    # configuration 3: one DCA layer
+    cfg = wl.CONFIGS[3]
+    co, so = wl.cand_offsets(cfg), wl.seq_offsets(cfg)
+    N = int(co[-1])
+    d = wl.dca_inputs(cfg, co, so)
+    plan = rocs.plan_create(dev(co), co)
+    Q, K, V, sod = dev(d["Q"]), dev(d["K"]), dev(d["V"]), dev(so)
+    O = torch.empty_like(Q)
+    t = time_call(lambda i: rocs.dca_attention(plan, Q, K, V, sod, out=O), reps=5)
+    pairs = float(np.sum(np.diff(co).astype(np.float64) * np.diff(so)))
+    flops = 4.0 * pairs * cfg.H * cfg.dh
+    nbytes = (2 * Q.numel() + 2 * K.numel()) * 2
+    out.append({"layer": "cfg3 dca_attention (R=64, L=2048, 8x64)", "N": N, "us": t * 1e6, "cand_per_s": N / t,
+                "tflops": flops / t / 1e12, "frac_tensor": flops / t / 1e12 / peaks["tflops_burst"],
+                "gbs": nbytes / t / 1e9, "exps_per_s": pairs * cfg.H / t})
+    del Q, K, V, O
+    # configuration 4: GLM interaction + compression
+    cfg = wl.CONFIGS[4]
+    co = wl.cand_offsets(cfg)
+    N = int(co[-1])
+    d = wl.glm_inputs(cfg, co)
+    plan4 = rocs.plan_create(dev(co), co)
+    XR, XC, W = dev(d["XR"]), dev(d["XC"]), dev(d["W"])
+    n = cfg.n_r + cfg.n_c
+    outs = {"OC": torch.empty((N, cfg.n_co, n), dtype=torch.bfloat16, device="cuda"),
+            "OR": torch.empty((cfg.R, cfg.n_ro, n), dtype=torch.bfloat16, device="cuda")}
+    ws = torch.empty(rocs.glm_interaction_workspace(plan4, cfg.n_r, cfg.n_c, cfg.n_co), dtype=torch.uint8, device="cuda")
+    t = time_call(lambda i: rocs.glm_interaction(plan4, XR, XC, W, cfg.n_ro, cfg.n_co, want_raw=False, workspace=ws,
+                                                 outs=outs), reps=10)
+    nbytes = XC.numel() * 2 + outs["OC"].numel() * 2 + XR.numel() * 2
+    flops = N * (2.0 * cfg.n_c * n * cfg.d_emb + 2.0 * cfg.n_co * cfg.n_c * n)
+    out.append({"layer": "cfg4 glm_interaction 32+16 x128, 48->16 compression (OC only)", "N": N, "us": t * 1e6,
+                "cand_per_s": N / t, "gbs": nbytes / t / 1e9, "frac_hbm": nbytes / t / 1e9 / peaks["hbm_gbs"],
+                "tflops": flops / t / 1e12,
+                "note": "input (537 MB) is larger than L2; same buffers every iteration"})
+    return out
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=1000)
+    ap.add_argument("--warmup", type=int, default=10)
+    ap.add_argument("--impl", default="rocs", choices=["rocs", "reference"])
+    ap.add_argument("--skip-extra", action="store_true", help="skip the attention / interaction side measurements")
+    ap.add_argument("--skip-cpu", action="store_true", help="skip the cpu_baseline leg")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3) if args.impl == "rocs" else args.warmup
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_rocs(args)
+
+
+if __name__ == "__main__":
+    main()

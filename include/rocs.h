@@ -1,0 +1,189 @@
+/*
+ * rocs.h -- C ABI of the B200 (sm_100a) In-Kernel Broadcast Optimization library.
+ *
+ * The library evaluates the candidate-side hot path of ROCS request-candidate layers:
+ * request tensors stay at batch size R (B_r in the paper), candidate tensors at batch
+ * size N (B_c), and each kernel resolves the request of a candidate inside the kernel
+ * (Section 4, "In-Kernel Broadcast Optimization"); nothing is replicated per candidate.
+ *
+ * Conventions
+ *   - Every pointer is a DEVICE pointer unless its name ends in _host.  The caller owns
+ *     all buffers; the library allocates only what a plan holds.
+ *   - Matrices are row-major, innermost dimension last.  `ld_*` are row strides in
+ *     ELEMENTS.  Every base pointer must be 16-byte aligned and every row stride must
+ *     be a multiple of 16 bytes (the memory-alignment rule of Section 4.2.4 made
+ *     explicit; rocs_padded_ld gives the zero-padded stride).
+ *   - Candidates of one request are stored consecutively: request r owns candidate
+ *     rows cand_offsets[r] .. cand_offsets[r+1]-1.  This is the index map m of
+ *     Section 4.1 in segment form.  Empty requests are legal.
+ *   - Work is enqueued on `stream` (a cudaStream_t, NULL = default stream) and the call
+ *     returns without synchronising, except where stated.
+ *   - Errors are return codes.  Arguments are validated before anything is enqueued: every
+ *     code except ROCS_ERR_CUDA means that the call launched nothing.
+ *   - dtype names the storage type of all X / W / Q / K / V / output tensors of a call.
+ *     ROCS_BF16: bf16 storage, fp32 accumulation (tensor cores where the shape allows),
+ *     softmax in fp32, results rounded to bf16 (nearest even).  ROCS_F32: fp32 storage
+ *     and plain fp32 FMA arithmetic.
+ *   - Results are run-to-run bitwise deterministic, and a candidate's output bits do not
+ *     depend on any other candidate's inputs (the GLM invariant, Eq. 1).
+ */
+#ifndef ROCS_H_
+#define ROCS_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+  ROCS_OK = 0,
+  ROCS_ERR_INVALID_ARG = -1, /* null pointer, negative or inconsistent size            */
+  ROCS_ERR_ALIGNMENT = -2,   /* base pointer or row stride not a multiple of 16 bytes  */
+  ROCS_ERR_UNSUPPORTED = -3, /* shape outside what the kernels handle                  */
+  ROCS_ERR_SEGMENTS = -4,    /* offsets not non-decreasing / wrong end points          */
+  ROCS_ERR_WORKSPACE = -5,   /* workspace NULL, misaligned or too small                */
+  ROCS_ERR_CUDA = -6,        /* a CUDA runtime or driver call failed                   */
+  ROCS_ERR_TIMEOUT = -7      /* a bounded device-side wait expired (see rocs_last_device_status) */
+} rocs_status_t;
+
+typedef enum { ROCS_BF16 = 0, ROCS_F32 = 1 } rocs_dtype_t;
+typedef enum { ROCS_ACT_NONE = 0, ROCS_ACT_RELU = 1 } rocs_act_t;
+
+/* Which kernels a ROCS_BF16 call may use.  AUTO picks the tcgen05 tensor-core kernels when
+ * the shape qualifies and the general kernels otherwise; GENERAL forces the general
+ * (CUDA-core, fp32 FMA) kernels, which accept every legal shape. */
+typedef enum { ROCS_PATH_AUTO = 0, ROCS_PATH_GENERAL = 1 } rocs_path_t;
+
+typedef struct rocs_plan rocs_plan_t; /* opaque; owned by the library */
+
+const char* rocs_status_string(rocs_status_t status);
+
+/* Smallest row stride (in elements) >= n whose byte size is a multiple of 16
+ * (Section 4.2.4, memory alignment). */
+int64_t rocs_padded_ld(int64_t n, rocs_dtype_t dtype);
+
+/* Process-wide kernel-path selector (default ROCS_PATH_AUTO).  Not thread-safe against
+ * concurrent calls of the compute entry points. */
+rocs_status_t rocs_set_path(rocs_path_t path);
+
+/*
+ * Segment plan (Section 4.1: the request-candidate map m).  Built once per batch and
+ * shared by every layer that uses the same cand_offsets.
+ *   R, N               number of requests and of candidates (N < 2^31)
+ *   cand_offsets       [R+1] device int32, non-decreasing, [0] = 0, [R] = N; must stay
+ *                      valid and unchanged for the plan's lifetime
+ *   cand_offsets_host  optional host copy of the same array.  When given, validation and
+ *                      tile planning use it and the call does not synchronise; when NULL
+ *                      the offsets are copied back from the device (the call synchronises
+ *                      `stream`).
+ * The plan owns device arrays of O(N + number of tiles) int32, allocated and freed in stream
+ * order on `stream` (cudaMallocAsync); use the plan on that stream, or order other streams
+ * behind it yourself.  Tile lists for a given number of rows per candidate are created on
+ * first use by the attention / interaction calls (one allocation + copy) and cached.
+ * Errors: INVALID_ARG, SEGMENTS, CUDA.
+ */
+rocs_status_t rocs_plan_create(rocs_plan_t** out, int32_t R, int64_t N,
+                               const int32_t* cand_offsets,
+                               const int32_t* cand_offsets_host, void* stream);
+rocs_status_t rocs_plan_destroy(rocs_plan_t* plan);
+
+/*
+ * GLM linear layer, candidate side, with the request half broadcast inside the kernel
+ * (Eq. 4 for two groups; decomposition of Section 4.1; Eq. 14; fused epilogue of
+ * Section 4.2.1):
+ *     Z   = X^R W_CR^T + bias                 once per request, fp32, in `workspace`
+ *     Y_i = act( Z[m_i] + X^C_i W_CC^T )      for every candidate i
+ *   XR   [R, d_req], ld_xr       request features   (ignored when d_req == 0)
+ *   XC   [N, d_cand], ld_xc      candidate features
+ *   W_CR [d_out, d_req], ld_wcr  request block of the masked weight row [W_CR | W_CC];
+ *   W_CC [d_out, d_cand], ld_wcc the two may alias one [d_out, d_req+d_cand] matrix
+ *                                (W_CR = W, W_CC = W + d_req, both strides d_req+d_cand)
+ *   bias [d_out] fp32 or NULL
+ *   Y    [N, d_out], ld_y        output, storage type `dtype`
+ *   workspace                    >= rocs_ikbo_linear_workspace(plan, d_out) bytes, 256-byte
+ *                                aligned; contents are overwritten; unused when d_req == 0
+ * d_req == 0 gives the plain one-group layer Y = act(X^C W_CC^T + bias).
+ * Errors: INVALID_ARG, ALIGNMENT, WORKSPACE, UNSUPPORTED, CUDA.
+ */
+size_t rocs_ikbo_linear_workspace(const rocs_plan_t* plan, int32_t d_out);
+rocs_status_t rocs_ikbo_linear(const rocs_plan_t* plan, rocs_dtype_t dtype, int32_t d_req,
+                               int32_t d_cand, int32_t d_out, const void* XR, int64_t ld_xr,
+                               const void* XC, int64_t ld_xc, const void* W_CR, int64_t ld_wcr,
+                               const void* W_CC, int64_t ld_wcc, const float* bias,
+                               rocs_act_t act, void* Y, int64_t ld_y, void* workspace,
+                               size_t workspace_bytes, void* stream);
+
+/*
+ * One-group linear layer Y = act(X W^T + bias) on M rows (Eq. 4 with a single group):
+ * the plain layers that follow a split layer, and request-side products at batch size R.
+ *   X [M, d_in], ld_x;  W [d_out, d_in], ld_w;  bias [d_out] fp32 or NULL;  Y [M, d_out], ld_y.
+ * Errors: INVALID_ARG, ALIGNMENT, UNSUPPORTED, CUDA.
+ */
+rocs_status_t rocs_linear(rocs_dtype_t dtype, int64_t M, int32_t d_in, int32_t d_out,
+                          const void* X, int64_t ld_x, const void* W, int64_t ld_w,
+                          const float* bias, rocs_act_t act, void* Y, int64_t ld_y,
+                          void* stream);
+
+/*
+ * Group-wise cross attention, candidate side (Eq. 13, second line; K/V sharing of
+ * Section 4.3.1): every query row of candidate i attends over the sequence of its own
+ * request m_i, whose keys and values exist once:
+ *     O[i,t,h,:] = sum_j softmax_j( scale * <Q[i,t,h,:], K[s_r + j, h, :]> ) V[s_r + j, h, :]
+ * with r = m_i, s_r = seq_offsets[r], j over the L_r = seq_offsets[r+1]-seq_offsets[r]
+ * positions of that request.  No mask, no dropout, no output projection.
+ *   Q [N, n_q, H, dh] dense;  K, V [T, H, dh] dense;  O [N, n_q, H, dh]
+ *   T            number of sequence rows in K and V; must equal seq_offsets[R] (T < 2^31)
+ *   seq_offsets  [R+1] device int32, non-decreasing, [0] = 0 (contents are not validated)
+ *   scale <= 0 selects 1/sqrt(dh)
+ *   dh * sizeof(element) must be a multiple of 16; dh <= 256
+ * A request with L_r = 0 yields zero rows.  `workspace` may be NULL when
+ * rocs_dca_attention_workspace returns 0.
+ * Errors: INVALID_ARG, ALIGNMENT, WORKSPACE, UNSUPPORTED, CUDA.
+ */
+size_t rocs_dca_attention_workspace(const rocs_plan_t* plan, int32_t n_q, int32_t H, int32_t dh);
+rocs_status_t rocs_dca_attention(const rocs_plan_t* plan, rocs_dtype_t dtype, int32_t n_q,
+                                 int32_t H, int32_t dh, float scale, const void* Q,
+                                 const void* K, const void* V, int64_t T,
+                                 const int32_t* seq_offsets, void* O, void* workspace,
+                                 size_t workspace_bytes, void* stream);
+
+/*
+ * GLM factorization machine for two groups (Eq. 9-10) with the optional ROCSified
+ * linear compression on the row axis (Eq. 5-6), n = n_r + n_c:
+ *     YR[r] = [ X^R_r X^R_r^T , 0 ]                         [R, n_r, n]   once per request
+ *     YC[i] = [ X^C_i X^R_{m_i}^T , X^C_i X^C_i^T ]         [N, n_c, n]
+ *     OR[r] = W_RR YR[r]                                    [R, n_ro, n]
+ *     OC[i] = W_CR YR[m_i] + W_CC YC[i]                     [N, n_co, n]
+ * where W = [[W_RR, *], [W_CR, W_CC]] is [n_ro + n_co, n] dense row-major and its
+ * upper-right block W[0:n_ro, n_r:n] is never read (the mask of Eq. 3).  The request
+ * term W_CR YR[r] is formed once per request (fp32, in `workspace`) and added to each
+ * candidate of r inside the candidate kernel.
+ *   XR [R, n_r, d] dense;  XC [N, n_c, d] dense;  d * sizeof(element) multiple of 16
+ *   W == NULL: no compression; OR_ and OC must be NULL, n_ro = n_co = 0
+ *   YR, YC: raw interaction blocks, either may be NULL (not written)
+ *   OR_, OC: compressed outputs, either may be NULL (not written)
+ *   workspace >= rocs_glm_interaction_workspace(...) bytes, 256-byte aligned
+ * Errors: INVALID_ARG, ALIGNMENT, WORKSPACE, UNSUPPORTED, CUDA.
+ */
+size_t rocs_glm_interaction_workspace(const rocs_plan_t* plan, int32_t n_r, int32_t n_c,
+                                      int32_t n_co);
+rocs_status_t rocs_glm_interaction(const rocs_plan_t* plan, rocs_dtype_t dtype, int32_t n_r,
+                                   int32_t n_c, int32_t d, const void* XR, const void* XC,
+                                   const void* W, int32_t n_ro, int32_t n_co, void* YR,
+                                   void* YC, void* OR_, void* OC, void* workspace,
+                                   size_t workspace_bytes, void* stream);
+
+/*
+ * Device-side status of the tensor-core kernels.  Their barrier waits are bounded; a wait
+ * that expires records a code in a device word instead of spinning forever and the kernel
+ * returns.  This call synchronises the device, reads the word, clears it and returns
+ * ROCS_OK or ROCS_ERR_TIMEOUT; *detail_host (optional) receives the raw word.
+ */
+rocs_status_t rocs_last_device_status(uint32_t* detail_host);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* ROCS_H_ */

@@ -1,0 +1,93 @@
+// Internal declarations shared by the translation units of librocs.so.
+#pragma once
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+
+#include <cstdint>
+#include <map>
+#include <mutex>
+#include <vector>
+
+#include "../../include/rocs.h"
+
+namespace rocs {
+
+// One unit of work of the attention / interaction kernels: `count` consecutive candidates
+// of request `req`, starting at candidate row `cand0`.  A tile never crosses a request.
+struct Tile {
+  int32_t req;
+  int32_t cand0;
+  int32_t count;
+  int32_t pad;
+};
+
+struct TileList {
+  Tile* dev = nullptr;
+  int32_t num = 0;
+};
+
+}  // namespace rocs
+
+struct rocs_plan {
+  int32_t R = 0;
+  int64_t N = 0;
+  const int32_t* cand_offsets = nullptr;  // device, borrowed
+  int32_t* row2req = nullptr;             // device [N], m_i of Section 4.1
+  std::vector<int32_t> offsets_host;      // [R+1]
+  mutable std::mutex mu;
+  mutable std::map<int32_t, rocs::TileList> tiles;  // key: candidates per tile
+  int device = 0;
+  cudaStream_t stream = nullptr;  // stream the plan was created on; its memory is freed there
+};
+
+namespace rocs {
+
+#define ROCS_CUDA_TRY(expr)                    \
+  do {                                         \
+    cudaError_t _e = (expr);                   \
+    if (_e != cudaSuccess) return ROCS_ERR_CUDA; \
+  } while (0)
+
+inline size_t elem_size(rocs_dtype_t dt) { return dt == ROCS_BF16 ? 2 : 4; }
+inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+inline size_t round_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+
+// Returns the cached tile list for `cands_per_tile`, building it on first use.
+rocs_status_t plan_tiles(const rocs_plan* plan, int32_t cands_per_tile, cudaStream_t stream,
+                         TileList* out);
+
+// ---- general (CUDA-core) kernels: simt_kernels.cu -------------------------------------
+// Y[i, :] = act(add[row2req ? row2req[i] : -, :] + X[i, :] W^T + bias).  out_f32 selects an
+// fp32 output regardless of the storage type (used for the request half Z).
+rocs_status_t simt_linear(rocs_dtype_t dt, int64_t M, int32_t d_in, int32_t d_out, const void* X,
+                          int64_t ld_x, const void* W, int64_t ld_w, const float* bias,
+                          const float* add, int64_t ld_add, const int32_t* row2req, int act,
+                          void* Y, int64_t ld_y, bool out_f32, cudaStream_t stream);
+rocs_status_t simt_dca(rocs_dtype_t dt, const rocs_plan* plan, int32_t n_q, int32_t H, int32_t dh,
+                       float scale, const void* Q, const void* K, const void* V,
+                       const int32_t* seq_offsets, void* O, cudaStream_t stream);
+rocs_status_t simt_glm(rocs_dtype_t dt, const rocs_plan* plan, int32_t n_r, int32_t n_c, int32_t d,
+                       const void* XR, const void* XC, const void* W, int32_t n_ro, int32_t n_co,
+                       void* YR, void* YC, void* OR_, void* OC, float* zr_workspace,
+                       cudaStream_t stream);
+
+// ---- tcgen05 tensor-core kernels (bf16): umma_*.cu -------------------------------------
+bool umma_linear_supported(int64_t M, int32_t d_in, int32_t d_out, int64_t ld_x, int64_t ld_w,
+                           int64_t ld_y, bool out_f32);
+rocs_status_t umma_linear(int64_t M, int32_t d_in, int32_t d_out, const void* X, int64_t ld_x,
+                          const void* W, int64_t ld_w, const float* bias, const float* add,
+                          int64_t ld_add, const int32_t* row2req, int act, void* Y, int64_t ld_y,
+                          bool out_f32, cudaStream_t stream);
+bool umma_dca_supported(int32_t n_q, int32_t H, int32_t dh);
+rocs_status_t umma_dca(const rocs_plan* plan, int32_t n_q, int32_t H, int32_t dh, float scale,
+                       const void* Q, const void* K, const void* V, const int32_t* seq_offsets,
+                       int64_t T, void* O, cudaStream_t stream);
+bool umma_glm_supported(int32_t n_r, int32_t n_c, int32_t d, int32_t n_ro, int32_t n_co);
+rocs_status_t umma_glm(const rocs_plan* plan, int32_t n_r, int32_t n_c, int32_t d, const void* XR,
+                       const void* XC, const void* W, int32_t n_ro, int32_t n_co, void* YC,
+                       void* OC, const float* zr_workspace, cudaStream_t stream);
+
+// Device status word written by bounded waits of the tensor-core kernels.
+uint32_t* device_status_word();
+
+}  // namespace rocs
