@@ -45,7 +45,8 @@ typedef enum {
   ROCS_ERR_SEGMENTS = -4,    /* offsets not non-decreasing / wrong end points          */
   ROCS_ERR_WORKSPACE = -5,   /* workspace NULL, misaligned or too small                */
   ROCS_ERR_CUDA = -6,        /* a CUDA runtime or driver call failed                   */
-  ROCS_ERR_TIMEOUT = -7      /* a bounded device-side wait expired (see rocs_last_device_status) */
+  ROCS_ERR_TIMEOUT = -7,     /* a bounded device-side wait expired (see rocs_last_device_status) */
+  ROCS_ERR_STATIC_LIMIT = -8 /* problem larger than the fixed scratch of rocs_ikbo_linear_static */
 } rocs_status_t;
 
 typedef enum { ROCS_BF16 = 0, ROCS_F32 = 1 } rocs_dtype_t;
@@ -114,6 +115,37 @@ rocs_status_t rocs_ikbo_linear(const rocs_plan_t* plan, rocs_dtype_t dtype, int3
                                const void* W_CC, int64_t ld_wcc, const float* bias,
                                rocs_act_t act, void* Y, int64_t ld_y, void* workspace,
                                size_t workspace_bytes, void* stream);
+
+/*
+ * The same layer for callers that cannot allocate device memory while they score a batch --
+ * a serving thread whose allocator is frozen after start-up, a plugin living inside another
+ * component's memory budget, a path where an allocation's possible synchronisation is not
+ * acceptable.  (The paper has no counterpart; this entry point exists for such hosts only.)
+ * It needs no plan and no workspace: the request half Z and the candidate->request map live in
+ * one fixed array inside the library image (5 MiB of device memory held by every GPU context
+ * that loads the library, until the process exits).  The call performs no cudaMalloc, cudaFree
+ * or other allocating routine.
+ *   Limits: R * d_out <= rocs_ikbo_linear_static_max_z_elems()      (1 Mi fp32 values)
+ *           N         <= rocs_ikbo_linear_static_max_candidates()   (256 Ki candidates)
+ *           beyond either, the call returns ROCS_ERR_STATIC_LIMIT and launches nothing.
+ *   cand_offsets [R+1] device int32 as for rocs_plan_create; its contents are not validated
+ *   (they live on the device).  d_req, d_cand, d_out > 0.  Other arguments as above.
+ *   The first call on a device looks up the array's device address (cudaGetSymbolAddress);
+ *   make that first call outside any stream capture.
+ *   All calls share the one array, and it keeps whatever the previous call left.  Each call
+ *   overwrites every word it later reads, so stale contents are harmless, but two calls whose
+ *   kernels overlap on the GPU (different streams, no ordering between them) race on it:
+ *   serialise them.
+ * Errors: INVALID_ARG, ALIGNMENT, STATIC_LIMIT, CUDA.
+ */
+size_t rocs_ikbo_linear_static_max_z_elems(void);
+size_t rocs_ikbo_linear_static_max_candidates(void);
+rocs_status_t rocs_ikbo_linear_static(rocs_dtype_t dtype, int32_t R, int64_t N,
+                                      const int32_t* cand_offsets, int32_t d_req, int32_t d_cand,
+                                      int32_t d_out, const void* XR, int64_t ld_xr, const void* XC,
+                                      int64_t ld_xc, const void* W_CR, int64_t ld_wcr,
+                                      const void* W_CC, int64_t ld_wcc, const float* bias,
+                                      rocs_act_t act, void* Y, int64_t ld_y, void* stream);
 
 /*
  * One-group linear layer Y = act(X W^T + bias) on M rows (Eq. 4 with a single group):

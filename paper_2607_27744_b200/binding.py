@@ -29,7 +29,8 @@ EXPORTS = [
     "rocs_status_string", "rocs_padded_ld", "rocs_set_path", "rocs_plan_create", "rocs_plan_destroy",
     "rocs_ikbo_linear_workspace", "rocs_ikbo_linear", "rocs_linear", "rocs_dca_attention_workspace",
     "rocs_dca_attention", "rocs_glm_interaction_workspace", "rocs_glm_interaction",
-    "rocs_last_device_status",
+    "rocs_last_device_status", "rocs_ikbo_linear_static", "rocs_ikbo_linear_static_max_z_elems",
+    "rocs_ikbo_linear_static_max_candidates",
 ]
 
 
@@ -69,6 +70,10 @@ def lib() -> ctypes.CDLL:
         L.rocs_glm_interaction.argtypes = [vp, ctypes.c_int, i32, i32, i32, vp, vp, vp, i32, i32, vp, vp, vp, vp,
                                            vp, sz, vp]
         L.rocs_last_device_status.argtypes = [ctypes.POINTER(ctypes.c_uint32)]
+        L.rocs_ikbo_linear_static_max_z_elems.restype = sz
+        L.rocs_ikbo_linear_static_max_candidates.restype = sz
+        L.rocs_ikbo_linear_static.argtypes = [ctypes.c_int, i32, i64, vp, i32, i32, i32, vp, i64, vp, i64, vp, i64,
+                                              vp, i64, vp, ctypes.c_int, vp, i64, vp]
         _lib = L
     return _lib
 
@@ -246,3 +251,19 @@ def glm_interaction(plan: Plan, XR: torch.Tensor, XC: torch.Tensor, W: Optional[
         _p(workspace), workspace.numel() if workspace is not None else 0, _stream())
     _check(code, "rocs_glm_interaction")
     return outs
+
+
+def ikbo_linear_static(cand_offsets: torch.Tensor, XR: torch.Tensor, XC: torch.Tensor, W_CR: torch.Tensor,
+                       W_CC: torch.Tensor, out: torch.Tensor, bias: Optional[torch.Tensor] = None,
+                       relu: bool = False) -> torch.Tensor:
+    """The split linear layer through ``rocs_ikbo_linear_static``: no plan, no workspace, and the call
+    allocates nothing -- for hosts that cannot call cudaMalloc while scoring.  The caller passes the
+    output tensor; scratch lives in a fixed array inside the library (limits: R * d_out <= 1 Mi,
+    N <= 256 Ki; calls share the array, so do not let two of them overlap on the GPU)."""
+    R, N = cand_offsets.numel() - 1, XC.shape[0]
+    code = lib().rocs_ikbo_linear_static(
+        _dtype_code(XC), R, N, _p(cand_offsets), XR.shape[1], XC.shape[1], W_CC.shape[0], _p(XR), _rows_2d(XR),
+        _p(XC), _rows_2d(XC), _p(W_CR), _rows_2d(W_CR), _p(W_CC), _rows_2d(W_CC), _p(bias),
+        ACT_RELU if relu else ACT_NONE, _p(out), _rows_2d(out), _stream())
+    _check(code, "rocs_ikbo_linear_static")
+    return out

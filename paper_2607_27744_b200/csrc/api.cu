@@ -83,6 +83,7 @@ const char* rocs_status_string(rocs_status_t s) {
     case ROCS_ERR_WORKSPACE: return "workspace missing, misaligned or too small";
     case ROCS_ERR_CUDA: return "CUDA call failed";
     case ROCS_ERR_TIMEOUT: return "bounded device-side wait expired";
+    case ROCS_ERR_STATIC_LIMIT: return "problem larger than the fixed scratch array of the no-allocation entry point";
   }
   return "unknown status";
 }
@@ -205,7 +206,7 @@ rocs_status_t rocs_ikbo_linear(const rocs_plan_t* plan, rocs_dtype_t dtype, int3
   if ((plan->N > 0 && (!Y || (d_cand > 0 && !XC))) || (d_cand > 0 && !W_CC) ||
       (d_req > 0 && (!W_CR || (plan->R > 0 && !XR))))
     return ROCS_ERR_INVALID_ARG;
-  if (!aligned16(Y) || !row_stride_ok(ld_y, d_out, dtype)) return ROCS_ERR_ALIGNMENT;
+  if (!aligned16(Y) || !aligned16(bias) || !row_stride_ok(ld_y, d_out, dtype)) return ROCS_ERR_ALIGNMENT;
   if (d_cand > 0 && (!aligned16(XC) || !aligned16(W_CC) || !row_stride_ok(ld_xc, d_cand, dtype) ||
                      !row_stride_ok(ld_wcc, d_cand, dtype)))
     return ROCS_ERR_ALIGNMENT;
@@ -237,7 +238,7 @@ rocs_status_t rocs_linear(rocs_dtype_t dtype, int64_t M, int32_t d_in, int32_t d
   if (dtype != ROCS_BF16 && dtype != ROCS_F32) return ROCS_ERR_INVALID_ARG;
   if (M < 0 || d_in <= 0 || d_out <= 0 || !X || !W || !Y) return ROCS_ERR_INVALID_ARG;
   if (act != ROCS_ACT_NONE && act != ROCS_ACT_RELU) return ROCS_ERR_INVALID_ARG;
-  if (!aligned16(X) || !aligned16(W) || !aligned16(Y) || !row_stride_ok(ld_x, d_in, dtype) ||
+  if (!aligned16(X) || !aligned16(W) || !aligned16(Y) || !aligned16(bias) || !row_stride_ok(ld_x, d_in, dtype) ||
       !row_stride_ok(ld_w, d_in, dtype) || !row_stride_ok(ld_y, d_out, dtype))
     return ROCS_ERR_ALIGNMENT;
   return linear_dispatch(dtype, M, d_in, d_out, X, ld_x, W, ld_w, bias, nullptr, 0, nullptr, act, Y,
