@@ -78,6 +78,12 @@ rocs_status_t umma_linear(int64_t M, int32_t d_in, int32_t d_out, const void* X,
                           const void* W, int64_t ld_w, const float* bias, const float* add,
                           int64_t ld_add, const int32_t* row2req, int act, void* Y, int64_t ld_y,
                           bool out_f32, cudaStream_t stream);
+// Weight-stationary variant for d_in <= 256 and bf16 output (umma_linear picks it when it applies).
+bool umma_linear_ws_supported(int64_t M, int32_t d_in, int32_t d_out, bool out_f32);
+rocs_status_t umma_linear_ws(int64_t M, int32_t d_in, int32_t d_out, const void* X, int64_t ld_x,
+                             const void* W, int64_t ld_w, const float* bias, const float* add,
+                             int64_t ld_add, const int32_t* row2req, int act, void* Y, int64_t ld_y,
+                             cudaStream_t stream);
 bool umma_dca_supported(int32_t n_q, int32_t H, int32_t dh);
 rocs_status_t umma_dca(const rocs_plan* plan, int32_t n_q, int32_t H, int32_t dh, float scale,
                        const void* Q, const void* K, const void* V, const int32_t* seq_offsets,

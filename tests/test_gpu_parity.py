@@ -58,6 +58,17 @@ def test_linear_bf16_ragged_segments_several_tiles(path, relu, bias):
     assert _run_linear(cfg, co, bias=bias, relu=relu, path=path) <= tol_for("bf16")
 
 
+@pytest.mark.parametrize("relu,bias", [(False, False), (True, True)])
+def test_linear_bf16_narrow_input_many_short_segments(relu, bias):
+    # N >= 512 with d_cand <= 256 takes the weight-stationary kernel; segments of 0..40 rows put
+    # several requests into every 32-row slab, so both the shared-memory and the global request
+    # rows are exercised; d_out = 328 leaves a ragged last column slice
+    counts = [(i * 7) % 41 for i in range(70)]
+    co = wl.offsets_from_counts(counts)
+    cfg = wl.CONFIGS[5].with_(R=len(counts), d_req=64, d_cand=200, d_out=328)
+    assert _run_linear(cfg, co, bias=bias, relu=relu) <= tol_for("bf16")
+
+
 @pytest.mark.parametrize("path", PATHS)
 def test_linear_bf16_odd_widths(path):
     co = wl.offsets_from_counts([5, 77, 1])
@@ -267,9 +278,9 @@ def test_candidate_isolation_is_bit_exact(path):
     """Eq. 1 on the GPU: perturb one candidate, every other candidate's output bits stay put;
     perturb one request, only its own segment moves.  Also run-to-run determinism."""
     rocs.set_path(path)
-    co = wl.offsets_from_counts([130, 1, 64, 200, 5])
-    so = wl.offsets_from_counts([150, 20, 128, 260, 64])
-    cfg = wl.CONFIGS[5].with_(R=5, d_req=128, d_cand=128, d_out=256, n_ro=4, n_co=4)
+    co = wl.offsets_from_counts([130, 1, 64, 300, 5, 150])
+    so = wl.offsets_from_counts([150, 20, 128, 260, 64, 33])
+    cfg = wl.CONFIGS[5].with_(R=6, d_req=128, d_cand=128, d_out=256, n_ro=4, n_co=4)
     plan = _plan(co)
     N = int(co[-1])
     j = int(co[3]) + 77           # a candidate in the middle of a tile
