@@ -300,7 +300,7 @@ def run_rocs(args):
     # ---- attention and interaction kernels on their own workloads ----------------------------
     extra = []
     if not args.skip_extra:
-        extra = bench_other_ops(torch, rocs, peaks, dev, time_call)
+        extra = bench_other_ops(torch, rocs, peaks, dev, time_call, args.extra.split(","))
 
     # ---- end to end from pinned host buffers ------------------------------------------------
     XR_h, XC_h, co_h = pinned(data["lin"]["XR"]), pinned(data["lin"]["XC"]), pinned(co)
@@ -351,9 +351,17 @@ def run_rocs(args):
     }))
 
 
-def bench_other_ops(torch, rocs, peaks, dev, time_call):
+def bench_other_ops(torch, rocs, peaks, dev, time_call, which=("dca", "glm")):
     """Attention on configuration 3 and interaction on configuration 4, one layer each."""
     out = []
+    if "dca" in which:
+        out.append(bench_dca(torch, rocs, peaks, dev, time_call))
+    if "glm" in which:
+        out.append(bench_glm(torch, rocs, peaks, dev, time_call))
+    return out
+
+
+def bench_dca(torch, rocs, peaks, dev, time_call):
     # configuration 3: one DCA layer
     cfg = wl.CONFIGS[3]
     co, so = wl.cand_offsets(cfg), wl.seq_offsets(cfg)
@@ -366,10 +374,12 @@ def bench_other_ops(torch, rocs, peaks, dev, time_call):
     pairs = float(np.sum(np.diff(co).astype(np.float64) * np.diff(so)))
     flops = 4.0 * pairs * cfg.H * cfg.dh
     nbytes = (2 * Q.numel() + 2 * K.numel()) * 2
-    out.append({"layer": "cfg3 dca_attention (R=64, L=2048, 8x64)", "N": N, "us": t * 1e6, "cand_per_s": N / t,
-                "tflops": flops / t / 1e12, "frac_tensor": flops / t / 1e12 / peaks["tflops_burst"],
-                "gbs": nbytes / t / 1e9, "exps_per_s": pairs * cfg.H / t})
-    del Q, K, V, O
+    return {"layer": "cfg3 dca_attention (R=64, L=2048, 8x64)", "N": N, "us": t * 1e6, "cand_per_s": N / t,
+            "tflops": flops / t / 1e12, "frac_tensor": flops / t / 1e12 / peaks["tflops_burst"],
+            "gbs": nbytes / t / 1e9, "exps_per_s": pairs * cfg.H / t}
+
+
+def bench_glm(torch, rocs, peaks, dev, time_call):
     # configuration 4: GLM interaction + compression
     cfg = wl.CONFIGS[4]
     co = wl.cand_offsets(cfg)
@@ -385,11 +395,10 @@ def bench_other_ops(torch, rocs, peaks, dev, time_call):
                                                  outs=outs), reps=10)
     nbytes = XC.numel() * 2 + outs["OC"].numel() * 2 + XR.numel() * 2
     flops = N * (2.0 * cfg.n_c * n * cfg.d_emb + 2.0 * cfg.n_co * cfg.n_c * n)
-    out.append({"layer": "cfg4 glm_interaction 32+16 x128, 48->16 compression (OC only)", "N": N, "us": t * 1e6,
-                "cand_per_s": N / t, "gbs": nbytes / t / 1e9, "frac_hbm": nbytes / t / 1e9 / peaks["hbm_gbs"],
-                "tflops": flops / t / 1e12,
-                "note": "input (537 MB) is larger than L2; same buffers every iteration"})
-    return out
+    return {"layer": "cfg4 glm_interaction 32+16 x128, 48->16 compression (OC only)", "N": N, "us": t * 1e6,
+            "cand_per_s": N / t, "gbs": nbytes / t / 1e9, "frac_hbm": nbytes / t / 1e9 / peaks["hbm_gbs"],
+            "tflops": flops / t / 1e12,
+            "note": "input (537 MB) is larger than L2; same buffers every iteration"}
 
 
 def main():
@@ -399,6 +408,7 @@ def main():
     ap.add_argument("--warmup", type=int, default=10)
     ap.add_argument("--impl", default="rocs", choices=["rocs", "reference"])
     ap.add_argument("--skip-extra", action="store_true", help="skip the attention / interaction side measurements")
+    ap.add_argument("--extra", default="dca,glm", help="which side measurements to run (dca, glm)")
     ap.add_argument("--skip-cpu", action="store_true", help="skip the cpu_baseline leg")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "rocs" else args.warmup

@@ -14,8 +14,12 @@
 // kernel is bound by reading X^C from HBM, the tensor pipe has slack).
 //
 // Persistent CTA, 10 warps: warp 0 TMA producer, warp 1 MMA issuer, two epilogue groups of four
-// warps that alternate tiles (each owns one TMEM accumulator and one staging area), so one group
-// drains and compresses a tile while the tensor pipe fills the other accumulator.
+// warps that alternate tiles (each owns one TMEM accumulator), so one group drains a tile while the
+// tensor pipe fills the other accumulator.  An epilogue warp owns 32 rows = 32 / n_c whole
+// candidates: it rounds their YC rows to bf16 into a private shared-memory buffer, copies them out
+// if the raw block is wanted, and forms OC = ZR + W_CC YC per candidate with warp-level
+// mma.sync m16n8k16 (W_CC fragments live in registers, YC fragments come through ldmatrix), so the
+// compression sees the same bf16 YC values a caller would read back.
 #include <algorithm>
 
 #include "rocs_internal.h"
@@ -27,7 +31,6 @@ namespace {
 using namespace ptx;
 
 constexpr int kThreads = 320;
-constexpr int kGroupThreads = 128;
 constexpr uint32_t kStatusGlm = 0x200;
 constexpr int kAccStride = 256;  // TMEM columns per accumulator
 
@@ -42,10 +45,6 @@ struct GlmParams {
   __nv_bfloat16* OC;       // [N, n_co, n] or null
   uint32_t* status;
 };
-
-__device__ __forceinline__ void group_sync(int g) {
-  asm volatile("bar.sync %0, %1;" ::"r"(1 + g), "r"(kGroupThreads) : "memory");
-}
 
 template <int NC>
 __global__ void __launch_bounds__(kThreads, 1)
@@ -67,6 +66,10 @@ glm_umma_kernel(const __grid_constant__ CUtensorMap map_xr, const __grid_constan
   const int32_t k_slices = p.d / 64;
   const int32_t slice_bytes = (p.n_r_pad + 128) * 128;
   const int32_t xr_bytes = p.n_r_pad * 128;
+  // Each CTA takes a contiguous run of tiles: consecutive tiles mostly share a request, so its
+  // X^R rows and ZR block stay hot in L1/L2, and the X^C stream of a CTA is sequential in HBM.
+  const int32_t t_begin = (int32_t)((int64_t)blockIdx.x * p.num_tiles / gridDim.x);
+  const int32_t t_end = (int32_t)((int64_t)(blockIdx.x + 1) * p.num_tiles / gridDim.x);
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < p.stages; ++s) {
@@ -97,7 +100,7 @@ glm_umma_kernel(const __grid_constant__ CUtensorMap map_xr, const __grid_constan
       prefetch_tensormap(&map_xc);
       uint32_t it = 0;
       bool ok = true;
-      for (int32_t t = blockIdx.x; t < p.num_tiles; t += gridDim.x, ++it) {
+      for (int32_t t = t_begin; t < t_end; ++t, ++it) {
         const Tile tile = p.tiles[t];
         const int s = it % p.stages;
         if (!mbar_wait(&empty[s], ((it / p.stages) & 1) ^ 1, abort_flag, p.status, kStatusGlm | 1)) { ok = false; break; }
@@ -122,7 +125,7 @@ glm_umma_kernel(const __grid_constant__ CUtensorMap map_xr, const __grid_constan
     const uint32_t idesc = umma_idesc_bf16(128, (uint32_t)(p.n_r_pad + 128), false, false);
     uint32_t it = 0;
     bool ok = true;
-    for (int32_t t = blockIdx.x; t < p.num_tiles; t += gridDim.x, ++it) {
+    for (int32_t t = t_begin; t < t_end; ++t, ++it) {
       const uint32_t acc = it & 1;
       const int s = it % p.stages;
       if (!mbar_wait(&tmem_empty[acc], ((it >> 1) & 1) ^ 1, abort_flag, p.status, kStatusGlm | 2)) { ok = false; break; }
@@ -149,38 +152,59 @@ glm_umma_kernel(const __grid_constant__ CUtensorMap map_xr, const __grid_constan
     }
   } else {
     // ------------------------------ epilogue groups ----------------------------------------
-    const int g = (warp - 2) / 4;         // group 0: warps 2-5, group 1: warps 6-9
-    const int q = warp % 4;               // TMEM lane quadrant
-    const int gt = (warp - 2) % 4 * 32 + lane;  // thread index inside the group, 0..127
-    const int row = q * 32 + lane;        // tile row = TMEM lane
-    float* yc = reinterpret_cast<float*>(staging + g * p.group_staging_bytes);  // [128][yc_stride]
-    float* wcc = yc + 128 * p.yc_stride;                                         // [n_c][n_co]
-    __nv_bfloat16* oc_s = reinterpret_cast<__nv_bfloat16*>(wcc + ((NC * p.n_co + 3) & ~3));  // [cands][n_co][n]
+    // Everything below is local to one warp: a warp owns 32 tile rows = 32 / NC whole candidates.
+    const int g = (warp - 2) / 4;  // group 0: warps 2-5, group 1: warps 6-9
+    const int q = warp % 4;        // TMEM lane quadrant = rows 32q .. 32q+31 of the tile
+    const int n8 = n / 8;
+    // bf16 copy of this warp's 32 rows of YC, row stride yc_stride bytes (16 mod 32: no conflicts)
+    uint8_t* yc_w = staging + g * p.group_staging_bytes + q * 32 * p.yc_stride;
+    uint8_t* my = yc_w + lane * p.yc_stride;
     const bool compress = p.W != nullptr && p.OC != nullptr;
+    // A fragments of W_CC for mma.m16n8k16 (rows = outputs o, padded to 16; cols = a, padded to
+    // 16 per K step): a0 = (g8, 2t..), a1 = (g8+8, 2t..), a2 = (g8, 2t+8..), a3 = (g8+8, 2t+8..)
+    constexpr int KS = (NC + 15) / 16;
+    uint32_t wa[KS][4];
+    const int g8 = lane / 4, t4 = lane % 4;
     if (compress) {
-      // W_CC, transposed to [a][o] so that one broadcast 16-byte load fetches four outputs.
-      for (int e = gt; e < NC * p.n_co; e += kGroupThreads) {
-        const int a = e / p.n_co, o = e % p.n_co;
-        wcc[e] = __bfloat162float(p.W[(int64_t)(p.n_ro + o) * n + p.n_r + a]);
-      }
+#pragma unroll
+      for (int ks = 0; ks < KS; ++ks)
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+          const int o = g8 + (i & 1) * 8, a0 = ks * 16 + 2 * t4 + (i >> 1) * 8;
+          __nv_bfloat16 lo = __float2bfloat16_rn(0.f), hi = lo;
+          if (o < p.n_co) {
+            const __nv_bfloat16* wrow = p.W + (int64_t)(p.n_ro + o) * n + p.n_r;
+            if (a0 < NC) lo = wrow[a0];
+            if (a0 + 1 < NC) hi = wrow[a0 + 1];
+          }
+          __nv_bfloat162 h2(lo, hi);
+          wa[ks][i] = *reinterpret_cast<uint32_t*>(&h2);
+        }
     }
-    group_sync(g);
     uint32_t it = 0;
-    for (int32_t t = blockIdx.x; t < p.num_tiles; t += gridDim.x, ++it) {
+    for (int32_t t = t_begin; t < t_end; ++t, ++it) {
       if ((int)(it & 1) != g) continue;
       const Tile tile = p.tiles[t];
       if (!mbar_wait(&tmem_full[g], (it >> 1) & 1, abort_flag, p.status, kStatusGlm | 4)) break;
       tc_fence_after_sync();
       const uint32_t t_row = tmem_base + g * kAccStride + ((uint32_t)(q * 32) << 16);
-      float* my = yc + row * p.yc_stride;
-      // request-candidate block: columns 0 .. n_r-1
+      // request-candidate block: columns 0 .. n_r-1 (n_r is a multiple of 8)
       for (int32_t c0 = 0; c0 < p.n_r; c0 += 16) {
         uint32_t v[16];
         tmem_ld_32x32b_x16(t_row + c0, v);
         tmem_ld_wait();
 #pragma unroll
-        for (int j = 0; j < 16; ++j)
-          if (c0 + j < p.n_r) my[c0 + j] = __uint_as_float(v[j]);
+        for (int h = 0; h < 2; ++h) {
+          if (c0 + 8 * h < p.n_r) {
+            uint4 w;
+            __nv_bfloat162 b2;
+            b2 = __floats2bfloat162_rn(__uint_as_float(v[8 * h + 0]), __uint_as_float(v[8 * h + 1])); w.x = *reinterpret_cast<uint32_t*>(&b2);
+            b2 = __floats2bfloat162_rn(__uint_as_float(v[8 * h + 2]), __uint_as_float(v[8 * h + 3])); w.y = *reinterpret_cast<uint32_t*>(&b2);
+            b2 = __floats2bfloat162_rn(__uint_as_float(v[8 * h + 4]), __uint_as_float(v[8 * h + 5])); w.z = *reinterpret_cast<uint32_t*>(&b2);
+            b2 = __floats2bfloat162_rn(__uint_as_float(v[8 * h + 6]), __uint_as_float(v[8 * h + 7])); w.w = *reinterpret_cast<uint32_t*>(&b2);
+            *reinterpret_cast<uint4*>(my + (c0 + 8 * h) * 2) = w;
+          }
+        }
       }
       // candidate-candidate block: the 32 x 32 diagonal block of this warp's rows, of which each
       // thread keeps the NC columns of its own candidate
@@ -192,81 +216,83 @@ glm_umma_kernel(const __grid_constant__ CUtensorMap map_xr, const __grid_constan
         __syncwarp();
         if (lane == 0) mbar_arrive(&tmem_empty[g]);
         const int sub = lane / NC;  // which candidate of the warp's 32 / NC this row belongs to
+        float x[NC];
 #pragma unroll
         for (int j = 0; j < NC; ++j) {
-          uint32_t x = v[j];
+          uint32_t xv = v[j];
 #pragma unroll
-          for (int s2 = 1; s2 < 32 / NC; ++s2) x = (sub == s2) ? v[s2 * NC + j] : x;
-          my[p.n_r + j] = __uint_as_float(x);
+          for (int s2 = 1; s2 < 32 / NC; ++s2) xv = (sub == s2) ? v[s2 * NC + j] : xv;
+          x[j] = __uint_as_float(xv);
+        }
+#pragma unroll
+        for (int j = 0; j < NC; j += 8) {
+          uint4 w;
+          __nv_bfloat162 b2;
+          b2 = __floats2bfloat162_rn(x[j + 0], x[j + 1]); w.x = *reinterpret_cast<uint32_t*>(&b2);
+          b2 = __floats2bfloat162_rn(x[j + 2], x[j + 3]); w.y = *reinterpret_cast<uint32_t*>(&b2);
+          b2 = __floats2bfloat162_rn(x[j + 4], x[j + 5]); w.z = *reinterpret_cast<uint32_t*>(&b2);
+          b2 = __floats2bfloat162_rn(x[j + 6], x[j + 7]); w.w = *reinterpret_cast<uint32_t*>(&b2);
+          *reinterpret_cast<uint4*>(my + (p.n_r + j) * 2) = w;
         }
       }
-      group_sync(g);
-      const int32_t rows_valid = tile.count * NC;
+      __syncwarp();
+      const int32_t rows_valid = min(32, tile.count * NC - q * 32);  // this warp's rows that are real
+      if (rows_valid <= 0) continue;
       if (p.YC != nullptr) {
-        // raw block, bf16, 8 values (16 bytes) per store; rows of the tile are contiguous in YC
-        __nv_bfloat16* dst = p.YC + (int64_t)tile.cand0 * NC * n;
-        const int32_t vecs = rows_valid * n / 8;
-        for (int32_t e = gt; e < vecs; e += kGroupThreads) {
-          const int32_t r0 = (e * 8) / n, c0 = (e * 8) % n;
-          const float* src = yc + r0 * p.yc_stride + c0;
-          uint4 w;
-          __nv_bfloat162 h;
-          h = __floats2bfloat162_rn(src[0], src[1]); w.x = *reinterpret_cast<uint32_t*>(&h);
-          h = __floats2bfloat162_rn(src[2], src[3]); w.y = *reinterpret_cast<uint32_t*>(&h);
-          h = __floats2bfloat162_rn(src[4], src[5]); w.z = *reinterpret_cast<uint32_t*>(&h);
-          h = __floats2bfloat162_rn(src[6], src[7]); w.w = *reinterpret_cast<uint32_t*>(&h);
-          *reinterpret_cast<uint4*>(dst + (int64_t)e * 8) = w;
+        // raw block: the warp's rows are contiguous in YC; 16-byte vectors
+        uint4* dst = reinterpret_cast<uint4*>(p.YC + ((int64_t)tile.cand0 * NC + q * 32) * n);
+        const int32_t vecs = rows_valid * n8;
+        for (int32_t e = lane; e < vecs; e += 32) {
+          const int32_t r0 = e / n8, c8 = e % n8;
+          dst[e] = *reinterpret_cast<const uint4*>(yc_w + r0 * p.yc_stride + c8 * 16);
         }
       }
       if (compress) {
-        // OC[c][o][b] = ZR[r][o][b] + sum_a W_CC[o][a] YC[c][a][b]; a thread owns up to four (c, b)
-        // pairs at a time and all outputs o of them, four outputs per pass.
+        // OC[c] (n_co x n) = ZR[r] + W_CC (n_co x NC) * YC[c] (NC x n) per candidate, on the warp-level
+        // tensor-core path (mma.sync m16n8k16): the product is tiny and needs no TMEM round trip.
         const float* zr = p.ZR + (int64_t)tile.req * p.n_co * n;
-        const int32_t pairs = tile.count * n;
-        for (int32_t e0 = 0; e0 < pairs; e0 += 4 * kGroupThreads) {
-          int32_t c[4], b[4];
-          bool on[4];
-#pragma unroll
-          for (int u = 0; u < 4; ++u) {
-            const int32_t e = e0 + u * kGroupThreads + gt;
-            on[u] = e < pairs;
-            c[u] = on[u] ? e / n : 0;
-            b[u] = on[u] ? e % n : 0;
-          }
-          for (int32_t o0 = 0; o0 < p.n_co; o0 += 4) {
-            float acc[4][4];
-#pragma unroll
-            for (int u = 0; u < 4; ++u)
-#pragma unroll
-              for (int oo = 0; oo < 4; ++oo)
-                acc[u][oo] = (on[u] && o0 + oo < p.n_co) ? __ldg(zr + (o0 + oo) * n + b[u]) : 0.f;
-#pragma unroll
-            for (int a = 0; a < NC; ++a) {
-              float w[4];
-#pragma unroll
-              for (int oo = 0; oo < 4; ++oo) w[oo] = (o0 + oo < p.n_co) ? wcc[a * p.n_co + o0 + oo] : 0.f;
-#pragma unroll
-              for (int u = 0; u < 4; ++u) {
-                const float y = yc[(c[u] * NC + a) * p.yc_stride + b[u]];
-#pragma unroll
-                for (int oo = 0; oo < 4; ++oo) acc[u][oo] = fmaf(w[oo], y, acc[u][oo]);
-              }
+        const int32_t cands = rows_valid / NC;
+        for (int32_t cl = 0; cl < cands; ++cl) {
+          __nv_bfloat16* oc = p.OC + ((int64_t)tile.cand0 + q * (32 / NC) + cl) * p.n_co * n;
+          for (int32_t j = 0; j < n8; ++j) {
+            float d0 = 0.f, d1 = 0.f, d2 = 0.f, d3 = 0.f;
+            const int32_t col = 8 * j + 2 * t4;
+            if (g8 < p.n_co) {
+              const float2 z = __ldg(reinterpret_cast<const float2*>(zr + g8 * n + col));
+              d0 = z.x; d1 = z.y;
+            }
+            if (g8 + 8 < p.n_co) {
+              const float2 z = __ldg(reinterpret_cast<const float2*>(zr + (g8 + 8) * n + col));
+              d2 = z.x; d3 = z.y;
             }
 #pragma unroll
-            for (int u = 0; u < 4; ++u)
-#pragma unroll
-              for (int oo = 0; oo < 4; ++oo)
-                if (on[u] && o0 + oo < p.n_co)
-                  oc_s[(c[u] * p.n_co + o0 + oo) * n + b[u]] = __float2bfloat16_rn(acc[u][oo]);
+            for (int ks = 0; ks < KS; ++ks) {
+              uint32_t b0, b1 = 0u;
+              const uint32_t addr = smem_u32(yc_w + (cl * NC + ks * 16 + (lane & 15)) * p.yc_stride + j * 16);
+              if constexpr (NC >= 16) {
+                asm volatile("ldmatrix.sync.aligned.m8n8.x2.trans.shared.b16 {%0, %1}, [%2];" : "=r"(b0), "=r"(b1) : "r"(addr));
+              } else {
+                const uint32_t addr8 = smem_u32(yc_w + (cl * NC + (lane & 7)) * p.yc_stride + j * 16);
+                asm volatile("ldmatrix.sync.aligned.m8n8.x1.trans.shared.b16 {%0}, [%1];" : "=r"(b0) : "r"(addr8));
+              }
+              asm volatile(
+                  "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0, %1, %2, %3}, {%4, %5, %6, %7}, {%8, %9}, "
+                  "{%0, %1, %2, %3};"
+                  : "+f"(d0), "+f"(d1), "+f"(d2), "+f"(d3)
+                  : "r"(wa[ks][0]), "r"(wa[ks][1]), "r"(wa[ks][2]), "r"(wa[ks][3]), "r"(b0), "r"(b1));
+            }
+            if (g8 < p.n_co) {
+              __nv_bfloat162 h2 = __floats2bfloat162_rn(d0, d1);
+              *reinterpret_cast<__nv_bfloat162*>(oc + g8 * n + col) = h2;
+            }
+            if (g8 + 8 < p.n_co) {
+              __nv_bfloat162 h2 = __floats2bfloat162_rn(d2, d3);
+              *reinterpret_cast<__nv_bfloat162*>(oc + (g8 + 8) * n + col) = h2;
+            }
           }
         }
-        group_sync(g);
-        const uint4* src = reinterpret_cast<const uint4*>(oc_s);
-        uint4* dst = reinterpret_cast<uint4*>(p.OC + (int64_t)tile.cand0 * p.n_co * n);
-        const int32_t vecs = tile.count * p.n_co * n / 8;
-        for (int32_t e = gt; e < vecs; e += kGroupThreads) dst[e] = src[e];
       }
-      group_sync(g);  // staging is reused by this group's next tile
+      __syncwarp();  // the row buffer is rewritten by this warp's next tile
     }
   }
 
@@ -300,10 +326,10 @@ GlmLayout glm_layout(int32_t n_r, int32_t n_c, int32_t d, int32_t n_co) {
   const int32_t n = n_r + n_c;
   L.n_r_pad = (n_r + 15) / 16 * 16;
   L.stage_bytes = (L.n_r_pad + 128) * d * 2;
-  L.yc_stride = n | 1;  // odd stride: row-per-thread writes hit distinct banks
-  const int32_t cands = 128 / n_c;
-  int32_t gs = 128 * L.yc_stride * 4 + ((n_c * n_co + 3) & ~3) * 4 + cands * n_co * n * 2;
-  L.group_staging_bytes = (gs + 127) & ~127;
+  // bf16 rows; a stride of 16 mod 32 bytes keeps 16-byte row writes and ldmatrix reads conflict free
+  L.yc_stride = (n * 2) % 32 == 0 ? n * 2 + 16 : n * 2;
+  (void)n_co;
+  L.group_staging_bytes = (128 * L.yc_stride + 127) & ~127;
   const int32_t fixed = 2 * L.group_staging_bytes + 512 + 1024;
   L.stages = std::min(6, (kMaxSmem - fixed) / L.stage_bytes);
   L.smem_bytes = L.stages * L.stage_bytes + fixed;
@@ -318,7 +344,7 @@ bool umma_glm_supported(int32_t n_r, int32_t n_c, int32_t d, int32_t n_ro, int32
   if (n_c != 8 && n_c != 16 && n_c != 32) return false;
   if (n_r < 1 || n_r > 128) return false;
   if (d % 64 != 0 || d < 64 || d > 256) return false;
-  if ((n_r + n_c) % 8 != 0) return false;
+  if (n_r % 8 != 0 || n_co > 16) return false;
   return glm_layout(n_r, n_c, d, n_co).ok;
 }
 
