@@ -67,6 +67,42 @@ rocs_status_t plan_tiles(const rocs_plan* plan, int32_t cands_per_tile, cudaStre
   return ROCS_OK;
 }
 
+rocs_status_t plan_dca_items(const rocs_plan* plan, int32_t cands_per_tile, int32_t heads, cudaStream_t stream,
+                             DcaItemList* out) {
+  if (cands_per_tile < 1 || cands_per_tile > 32767 || heads < 1 || heads > 65535) return ROCS_ERR_INVALID_ARG;
+  std::lock_guard<std::mutex> lock(plan->mu);
+  const int64_t key = (int64_t)cands_per_tile * 65536 + heads;
+  auto it = plan->dca_items.find(key);
+  if (it != plan->dca_items.end()) {
+    *out = it->second;
+    return ROCS_OK;
+  }
+  std::vector<DcaItem> host;
+  for (int32_t r = 0; r < plan->R; ++r) {
+    const int32_t c_begin = plan->offsets_host[r], c_end = plan->offsets_host[r + 1];
+    if (c_begin == c_end) continue;
+    for (int32_t h = 0; h < heads; ++h)
+      for (int32_t c = c_begin; c < c_end; c += 2 * cands_per_tile) {
+        const int32_t a = std::min(cands_per_tile, c_end - c);
+        const int32_t b = std::min(cands_per_tile, c_end - c - a);
+        host.push_back(DcaItem{r, c, (int16_t)a, (int16_t)b, h});
+      }
+  }
+  DcaItemList il;
+  il.num = (int32_t)host.size();
+  if (il.num > 0) {
+    ROCS_CUDA_TRY(cudaMallocAsync((void**)&il.dev, sizeof(DcaItem) * host.size(), stream));
+    if (cudaMemcpyAsync(il.dev, host.data(), sizeof(DcaItem) * host.size(), cudaMemcpyHostToDevice, stream) !=
+        cudaSuccess) {
+      cudaFreeAsync(il.dev, stream);
+      return ROCS_ERR_CUDA;
+    }
+  }
+  plan->dca_items[key] = il;
+  *out = il;
+  return ROCS_OK;
+}
+
 }  // namespace rocs
 
 using namespace rocs;
@@ -171,6 +207,8 @@ rocs_status_t rocs_plan_destroy(rocs_plan_t* plan) {
   // Freed in stream order behind whatever the caller enqueued on the plan's stream.
   if (plan->row2req && cudaFreeAsync(plan->row2req, plan->stream) != cudaSuccess) st = ROCS_ERR_CUDA;
   for (auto& kv : plan->tiles)
+    if (kv.second.dev && cudaFreeAsync(kv.second.dev, plan->stream) != cudaSuccess) st = ROCS_ERR_CUDA;
+  for (auto& kv : plan->dca_items)
     if (kv.second.dev && cudaFreeAsync(kv.second.dev, plan->stream) != cudaSuccess) st = ROCS_ERR_CUDA;
   delete plan;
   return st;

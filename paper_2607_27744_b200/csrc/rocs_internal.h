@@ -26,6 +26,21 @@ struct TileList {
   int32_t num = 0;
 };
 
+// One unit of work of the tensor-core attention kernel: one head of up to two consecutive tiles
+// (A and B) of the same request, which then share every K/V block that is loaded.
+struct DcaItem {
+  int32_t req;
+  int32_t cand0;    // first candidate of tile A; tile B starts at cand0 + count_a
+  int16_t count_a;  // candidates in tile A (>= 1)
+  int16_t count_b;  // candidates in tile B (0 = no second tile)
+  int32_t head;
+};
+
+struct DcaItemList {
+  DcaItem* dev = nullptr;
+  int32_t num = 0;
+};
+
 }  // namespace rocs
 
 struct rocs_plan {
@@ -36,6 +51,7 @@ struct rocs_plan {
   std::vector<int32_t> offsets_host;      // [R+1]
   mutable std::mutex mu;
   mutable std::map<int32_t, rocs::TileList> tiles;  // key: candidates per tile
+  mutable std::map<int64_t, rocs::DcaItemList> dca_items;  // key: candidates per tile * 65536 + heads
   int device = 0;
   cudaStream_t stream = nullptr;  // stream the plan was created on; its memory is freed there
 };
@@ -55,6 +71,10 @@ inline size_t round_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 // Returns the cached tile list for `cands_per_tile`, building it on first use.
 rocs_status_t plan_tiles(const rocs_plan* plan, int32_t cands_per_tile, cudaStream_t stream,
                          TileList* out);
+
+// Work items for the attention kernel, ordered request, head, tile pair; cached in the plan.
+rocs_status_t plan_dca_items(const rocs_plan* plan, int32_t cands_per_tile, int32_t heads, cudaStream_t stream,
+                             DcaItemList* out);
 
 // ---- general (CUDA-core) kernels: simt_kernels.cu -------------------------------------
 // Y[i, :] = act(add[row2req ? row2req[i] : -, :] + X[i, :] W^T + bias).  out_f32 selects an

@@ -1,5 +1,411 @@
+// Group-wise cross attention, candidate side (Eq. 13), with the request's K/V shared inside the
+// kernel (Section 4.3.1):  O[i,t,h,:] = softmax_j(scale <Q[i,t,h,:], K[r,j,h,:]>) V[r,j,h,:],  r = m_i.
+//
+// Candidates of one request are stacked in the tile M dimension: a work item is one head of up to
+// TWO 128-row query tiles (A and B) of the same request, so every 128-key block of K and V is loaded
+// once and used by 256 query rows.  K/V are addressed per request through seq_offsets; nothing is
+// replicated per candidate.
+//
+// One persistent CTA per SM, 10 warps:
+//   warp 0     TMA producer: Q tiles of the item, then (K_j, V_j) blocks through a ring
+//   warp 1     tcgen05.mma issuer:  S_X = Q_X K_j^T  (128x128x64)  and  O_X = P_X V_j  (128x64x128)
+//   warps 2-5  softmax group A,  warps 6-9  softmax group B: each thread owns one query row:
+//              TMEM -> registers, running max and sum in fp32 (exp2 on scaled scores), P rounded to
+//              bf16 into shared memory (the A operand of the second MMA), O accumulated in registers
+//              across key blocks (O = O * alpha + P V), final 1/sum, bf16 store.
+// The two groups run half a phase apart, so while one waits for its next S tile the other keeps the
+// exponential unit busy.  Every row's arithmetic depends only on that row and its request's K/V.
+#include <algorithm>
+
 #include "rocs_internal.h"
+#include "sm100_ptx.cuh"
+
 namespace rocs {
-bool umma_dca_supported(int32_t, int32_t, int32_t) { return false; }
-rocs_status_t umma_dca(const rocs_plan*, int32_t, int32_t, int32_t, float, const void*, const void*, const void*, const int32_t*, int64_t, void*, cudaStream_t) { return ROCS_ERR_UNSUPPORTED; }
+namespace {
+
+using namespace ptx;
+
+constexpr int DH = 64;            // head dimension handled here (128-byte rows)
+constexpr int BQ = 128;           // query rows per tile
+constexpr int BKV = 128;          // keys per block
+constexpr int kThreads = 320;
+constexpr int kKvStages = 3;
+constexpr int kQBytes = BQ * DH * 2;          // 16 KB
+constexpr int kKvStageBytes = 2 * BKV * DH * 2;  // K block + V block = 32 KB
+constexpr int kPBytes = BQ * BKV * 2;         // 32 KB per side
+constexpr int kSmemBytes = 2 * kQBytes + kKvStages * kKvStageBytes + 2 * kPBytes + 256 + 1024;
+constexpr uint32_t kStatusDca = 0x400;
+constexpr int kSideTmemStride = 256;  // side A: columns 0.., side B: columns 256..
+constexpr int kOColOffset = 128;      // S in [0, 128), O block in [128, 192) of the side
+
+struct DcaParams {
+  const DcaItem* items;
+  int32_t num_items;
+  int32_t n_q, H;
+  float scale_log2e;  // scale * log2(e)
+  const int32_t* seq_offsets;
+  __nv_bfloat16* O;
+  int64_t n_rows;     // N * n_q
+  uint32_t* status;
+};
+
+__device__ __forceinline__ float ex2(float x) {
+  float y;
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
 }
+
+__global__ void __launch_bounds__(kThreads, 1)
+dca_umma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
+                const __grid_constant__ CUtensorMap map_v, const DcaParams p) {
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+  uint8_t* q_smem = smem;                              // [2][128][64] bf16
+  uint8_t* kv_smem = q_smem + 2 * kQBytes;             // [stages][K 16 KB | V 16 KB]
+  uint8_t* p_smem = kv_smem + kKvStages * kKvStageBytes;  // [2][2 x (128 x 64)] bf16, K-major swizzled
+  uint64_t* q_full = reinterpret_cast<uint64_t*>(p_smem + 2 * kPBytes);
+  uint64_t* item_done = q_full + 1;
+  uint64_t* item_start = item_done + 1;
+  uint64_t* kv_full = item_start + 1;
+  uint64_t* kv_empty = kv_full + kKvStages;
+  uint64_t* s_full = kv_empty + kKvStages;   // [2]
+  uint64_t* p_full = s_full + 2;             // [2]
+  uint64_t* o_full = p_full + 2;             // [2]
+  uint64_t* drain = o_full + 2;
+  uint32_t* tmem_ptr = reinterpret_cast<uint32_t*>(drain + 1);
+  AbortFlag* abort_flag = reinterpret_cast<AbortFlag*>(tmem_ptr + 1);
+
+  const int warp = threadIdx.x / 32, lane = threadIdx.x % 32;
+
+  if (threadIdx.x == 0) {
+    mbar_init(q_full, 1);
+    mbar_init(item_done, 8);
+    mbar_init(item_start, 1);
+    for (int s = 0; s < kKvStages; ++s) {
+      mbar_init(&kv_full[s], 1);
+      mbar_init(&kv_empty[s], 1);
+    }
+    for (int x = 0; x < 2; ++x) {
+      mbar_init(&s_full[x], 1);
+      mbar_init(&p_full[x], 4);
+      mbar_init(&o_full[x], 1);
+    }
+    mbar_init(drain, 1);
+    abort_flag->v = 0;
+    fence_mbar_init();
+  }
+  if (warp == 1) {
+    tmem_alloc(tmem_ptr, 512);
+    tmem_relinquish();
+  }
+  tc_fence_before_sync();
+  __syncthreads();
+  tc_fence_after_sync();
+  const uint32_t tmem_base = *tmem_ptr;
+  const int32_t row_width = p.H * DH;  // elements per query / key row over all heads
+
+  if (warp == 0) {
+    // ------------------------------ TMA producer ------------------------------------------
+    if (lane == 0) {
+      prefetch_tensormap(&map_q);
+      prefetch_tensormap(&map_k);
+      prefetch_tensormap(&map_v);
+      uint32_t kv_it = 0, n_item = 0;
+      bool ok = true;
+      for (int32_t i = blockIdx.x; i < p.num_items && ok; i += gridDim.x, ++n_item) {
+        const DcaItem item = p.items[i];
+        const int32_t s0 = p.seq_offsets[item.req];
+        const int32_t L = p.seq_offsets[item.req + 1] - s0;
+        // Q buffers are free once both softmax groups have finished the previous item
+        if (!mbar_wait(item_done, (n_item & 1) ^ 1, abort_flag, p.status, kStatusDca | 1)) { ok = false; break; }
+        mbar_arrive(item_start);  // the softmax warps may enter this item (keeps them in step, also when idle)
+        if (L == 0) continue;
+        const int32_t sides = item.count_b > 0 ? 2 : 1;
+        mbar_expect_tx(q_full, sides * kQBytes);
+        tma_load_2d(q_smem, &map_q, q_full, item.head * DH, item.cand0 * p.n_q);
+        if (sides == 2) tma_load_2d(q_smem + kQBytes, &map_q, q_full, item.head * DH, (item.cand0 + item.count_a) * p.n_q);
+        const int32_t nblk = (L + BKV - 1) / BKV;
+        for (int32_t j = 0; j < nblk; ++j, ++kv_it) {
+          const int s = kv_it % kKvStages;
+          if (!mbar_wait(&kv_empty[s], ((kv_it / kKvStages) & 1) ^ 1, abort_flag, p.status, kStatusDca | 2)) { ok = false; break; }
+          uint8_t* st = kv_smem + s * kKvStageBytes;
+          mbar_expect_tx(&kv_full[s], kKvStageBytes);
+          tma_load_2d(st, &map_k, &kv_full[s], item.head * DH, s0 + j * BKV);
+          tma_load_2d(st + BKV * DH * 2, &map_v, &kv_full[s], item.head * DH, s0 + j * BKV);
+        }
+      }
+      if (!ok) {
+        for (int s = 0; s < kKvStages; ++s) {
+          const uint32_t n_issued = kv_it / kKvStages + (((int)(kv_it % kKvStages) > s) ? 1 : 0);
+          if (n_issued == 0) continue;
+          const uint64_t t0 = globaltimer_ns();
+          while (!mbar_try_wait(&kv_full[s], (n_issued - 1) & 1) && globaltimer_ns() - t0 < kWaitLimitNs) {}
+        }
+      }
+    }
+  } else if (warp == 1) {
+    // ------------------------------ MMA issuer ---------------------------------------------
+    constexpr uint32_t idesc_s = umma_idesc_bf16(BQ, BKV, false, false);  // S = Q K^T, both K-major
+    constexpr uint32_t idesc_o = umma_idesc_bf16(BQ, DH, false, true);    // O = P V, V is MN-major
+    uint32_t kv_it = 0, n_work = 0;           // n_work: items that had keys (phase of q_full)
+    uint32_t cnt_p[2] = {0, 0};               // phases of p_full per side
+    bool ok = true;
+    auto issue_s = [&](int side, int stage) {
+      const uint32_t d = tmem_base + side * kSideTmemStride;
+      const uint64_t a_desc = smem_desc_sw128(smem_u32(q_smem + side * kQBytes), 1024, 16);
+      const uint64_t b_desc = smem_desc_sw128(smem_u32(kv_smem + stage * kKvStageBytes), 1024, 16);
+#pragma unroll
+      for (int k = 0; k < DH / 16; ++k) umma_ss(d, a_desc + 2 * k, b_desc + 2 * k, idesc_s, k != 0 ? 1u : 0u);
+      umma_commit(&s_full[side]);
+    };
+    auto issue_pv = [&](int side, int stage) {
+      const uint32_t d = tmem_base + side * kSideTmemStride + kOColOffset;
+      const uint32_t p_addr = smem_u32(p_smem + side * kPBytes);
+      const uint32_t v_addr = smem_u32(kv_smem + stage * kKvStageBytes + BKV * DH * 2);
+#pragma unroll
+      for (int k = 0; k < BKV / 16; ++k) {
+        // P: K-major, two 64-key blocks of 16 KB, 32 bytes per 16 keys inside a block
+        const uint64_t a_desc = smem_desc_sw128(p_addr + (k / 4) * (BQ * 128) + (k % 4) * 32, 1024, 16);
+        // V: rows are keys (K), 128 bytes = 64 head dims (N): 16 keys = 2048 bytes further on
+        const uint64_t b_desc = smem_desc_sw128(v_addr + k * 16 * 128, 1024, 16);
+        umma_ss(d, a_desc, b_desc, idesc_o, k != 0 ? 1u : 0u);
+      }
+      umma_commit(&o_full[side]);
+    };
+    for (int32_t i = blockIdx.x; i < p.num_items && ok; i += gridDim.x) {
+      const DcaItem item = p.items[i];
+      const int32_t L = p.seq_offsets[item.req + 1] - p.seq_offsets[item.req];
+      if (L == 0) continue;
+      const int32_t sides = item.count_b > 0 ? 2 : 1;
+      const int32_t nblk = (L + BKV - 1) / BKV;
+      if (!mbar_wait(q_full, n_work & 1, abort_flag, p.status, kStatusDca | 3)) { ok = false; break; }
+      ++n_work;
+      // first key block: S for both sides
+      if (!mbar_wait(&kv_full[kv_it % kKvStages], (kv_it / kKvStages) & 1, abort_flag, p.status, kStatusDca | 4)) { ok = false; break; }
+      tc_fence_after_sync();
+      if (lane == 0)
+        for (int x = 0; x < sides; ++x) issue_s(x, kv_it % kKvStages);
+      __syncwarp();
+      for (int32_t j = 0; j < nblk && ok; ++j, ++kv_it) {
+        const int stage = kv_it % kKvStages;
+        const int next_stage = (kv_it + 1) % kKvStages;
+        if (j + 1 < nblk) {
+          if (!mbar_wait(&kv_full[next_stage], ((kv_it + 1) / kKvStages) & 1, abort_flag, p.status, kStatusDca | 5)) { ok = false; break; }
+        }
+        for (int x = 0; x < sides; ++x) {
+          // P_j of this side is in shared memory and its S tile has been read
+          if (!mbar_wait(&p_full[x], cnt_p[x] & 1, abort_flag, p.status, kStatusDca | 6)) { ok = false; break; }
+          ++cnt_p[x];
+          tc_fence_after_sync();
+          if (lane == 0) {
+            issue_pv(x, stage);
+            if (j + 1 < nblk) issue_s(x, next_stage);
+          }
+          __syncwarp();
+        }
+        if (ok && lane == 0) umma_commit(&kv_empty[stage]);  // K_j and V_j are no longer needed
+        __syncwarp();
+      }
+    }
+    if (!ok && lane == 0) {
+      umma_commit(drain);
+      const uint64_t t0 = globaltimer_ns();
+      while (!mbar_try_wait(drain, 0) && globaltimer_ns() - t0 < kWaitLimitNs) {}
+    }
+  } else {
+    // ------------------------------ softmax groups -----------------------------------------
+    const int side = (warp - 2) / 4;
+    const int q = warp % 4;                 // TMEM lane quadrant
+    const int row = q * 32 + lane;          // query row of the tile = TMEM lane
+    const uint32_t t_s = tmem_base + side * kSideTmemStride + ((uint32_t)(q * 32) << 16);
+    const uint32_t t_o = t_s + kOColOffset;
+    uint8_t* p_row = p_smem + side * kPBytes + row * 128;
+    uint32_t cnt_s = 0, cnt_o = 0, n_item = 0;
+    for (int32_t i = blockIdx.x; i < p.num_items; i += gridDim.x, ++n_item) {
+      if (!mbar_wait(item_start, n_item & 1, abort_flag, p.status, kStatusDca | 10)) break;
+      const DcaItem item = p.items[i];
+      const int32_t L = p.seq_offsets[item.req + 1] - p.seq_offsets[item.req];
+      const int32_t my_count = side == 0 ? item.count_a : item.count_b;
+      const int32_t cand_first = side == 0 ? item.cand0 : item.cand0 + item.count_a;
+      const int32_t rows_valid = my_count * p.n_q;
+      __nv_bfloat16* out = p.O + ((int64_t)cand_first * p.n_q + row) * row_width + item.head * DH;
+      bool aborted = false;
+      float o_reg[DH];
+#pragma unroll
+      for (int e = 0; e < DH; ++e) o_reg[e] = 0.f;
+      float m_run = -INFINITY, l_run = 0.f, alpha_pending = 0.f;
+      if (my_count > 0 && L > 0) {
+        const int32_t nblk = (L + BKV - 1) / BKV;
+        for (int32_t j = 0; j < nblk; ++j) {
+          const int32_t valid = min(BKV, L - j * BKV);  // keys of this block that exist
+          if (!mbar_wait(&s_full[side], cnt_s & 1, abort_flag, p.status, kStatusDca | 7)) { aborted = true; break; }
+          ++cnt_s;
+          tc_fence_after_sync();
+          // pass 1: row maximum of the scaled scores
+          float mx = -INFINITY;
+#pragma unroll 1
+          for (int c = 0; c < BKV; c += 32) {
+            uint32_t v[32];
+            tmem_ld_32x32b_x32(t_s + c, v);
+            tmem_ld_wait();
+#pragma unroll
+            for (int e = 0; e < 32; ++e) {
+              const float s = __uint_as_float(v[e]) * p.scale_log2e;
+              mx = fmaxf(mx, (c + e < valid) ? s : -INFINITY);
+            }
+          }
+          const float m_new = fmaxf(m_run, mx);
+          const float alpha = ex2(m_run - m_new);  // 0 for the first block (m_run = -inf)
+          // fold the previous block's P V into the running output; this also tells us that the MMA
+          // has finished reading the previous P from shared memory
+          if (j > 0) {
+            if (!mbar_wait(&o_full[side], cnt_o & 1, abort_flag, p.status, kStatusDca | 8)) { aborted = true; break; }
+            ++cnt_o;
+            tc_fence_after_sync();
+#pragma unroll
+            for (int c = 0; c < DH; c += 32) {
+              uint32_t v[32];
+              tmem_ld_32x32b_x32(t_o + c, v);
+              tmem_ld_wait();
+#pragma unroll
+              for (int e = 0; e < 32; ++e) o_reg[c + e] = fmaf(o_reg[c + e], alpha_pending, __uint_as_float(v[e]));
+            }
+          }
+          alpha_pending = alpha;
+          m_run = m_new;
+          // pass 2: P = exp2(s - m), row sum, bf16 P into the swizzled K-major operand layout
+          float sum = 0.f;
+#pragma unroll 1
+          for (int c = 0; c < BKV; c += 32) {
+            uint32_t v[32];
+            tmem_ld_32x32b_x32(t_s + c, v);
+            tmem_ld_wait();
+            uint32_t packed[16];
+#pragma unroll
+            for (int e = 0; e < 32; e += 2) {
+              float p0 = ex2(fmaf(__uint_as_float(v[e]), p.scale_log2e, -m_new));
+              float p1 = ex2(fmaf(__uint_as_float(v[e + 1]), p.scale_log2e, -m_new));
+              p0 = (c + e < valid) ? p0 : 0.f;
+              p1 = (c + e + 1 < valid) ? p1 : 0.f;
+              sum += p0 + p1;
+              __nv_bfloat162 h2 = __floats2bfloat162_rn(p0, p1);
+              packed[e / 2] = *reinterpret_cast<uint32_t*>(&h2);
+            }
+            // 32 keys = four 16-byte chunks of this row inside the 64-key block c / 64
+            uint8_t* blk = p_row + (c / 64) * (BQ * 128);
+#pragma unroll
+            for (int u = 0; u < 4; ++u) {
+              const int chunk = (c % 64) / 8 + u;
+              *reinterpret_cast<uint4*>(blk + ((chunk ^ (row & 7)) << 4)) =
+                  make_uint4(packed[4 * u], packed[4 * u + 1], packed[4 * u + 2], packed[4 * u + 3]);
+            }
+          }
+          l_run = l_run * alpha + sum;
+          fence_proxy_async_smem();
+          tc_fence_before_sync();
+          __syncwarp();
+          if (lane == 0) mbar_arrive(&p_full[side]);
+        }
+        if (!aborted) {
+          if (!mbar_wait(&o_full[side], cnt_o & 1, abort_flag, p.status, kStatusDca | 9)) {
+            aborted = true;
+          } else {
+            ++cnt_o;
+            tc_fence_after_sync();
+#pragma unroll
+            for (int c = 0; c < DH; c += 32) {
+              uint32_t v[32];
+              tmem_ld_32x32b_x32(t_o + c, v);
+              tmem_ld_wait();
+#pragma unroll
+              for (int e = 0; e < 32; ++e) o_reg[c + e] = fmaf(o_reg[c + e], alpha_pending, __uint_as_float(v[e]));
+            }
+          }
+        }
+      }
+      if (aborted) break;
+      if (row < rows_valid) {
+        const float inv = (L > 0) ? 1.f / l_run : 0.f;
+#pragma unroll
+        for (int c = 0; c < DH; c += 8) {
+          uint4 w;
+          __nv_bfloat162 h2;
+          h2 = __floats2bfloat162_rn(o_reg[c + 0] * inv, o_reg[c + 1] * inv); w.x = *reinterpret_cast<uint32_t*>(&h2);
+          h2 = __floats2bfloat162_rn(o_reg[c + 2] * inv, o_reg[c + 3] * inv); w.y = *reinterpret_cast<uint32_t*>(&h2);
+          h2 = __floats2bfloat162_rn(o_reg[c + 4] * inv, o_reg[c + 5] * inv); w.z = *reinterpret_cast<uint32_t*>(&h2);
+          h2 = __floats2bfloat162_rn(o_reg[c + 6] * inv, o_reg[c + 7] * inv); w.w = *reinterpret_cast<uint32_t*>(&h2);
+          *reinterpret_cast<uint4*>(out + c) = w;
+        }
+      }
+      tc_fence_before_sync();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(item_done);
+    }
+  }
+
+  tc_fence_before_sync();
+  __syncthreads();
+  if (warp == 1) {
+    tc_fence_after_sync();
+    tmem_dealloc(tmem_base, 512);
+  }
+}
+
+int sm_count_dca() {
+  static int n = 0;
+  if (n == 0) {
+    int dev = 0;
+    cudaGetDevice(&dev);
+    cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev);
+  }
+  return n;
+}
+
+}  // namespace
+
+bool umma_dca_supported(int32_t n_q, int32_t H, int32_t dh) {
+  return dh == DH && n_q >= 1 && n_q <= BQ && H >= 1 && H <= 65535;
+}
+
+rocs_status_t umma_dca(const rocs_plan* plan, int32_t n_q, int32_t H, int32_t dh, float scale, const void* Q,
+                       const void* K, const void* V, const int32_t* seq_offsets, int64_t T, void* O,
+                       cudaStream_t stream) {
+  (void)dh;
+  if (plan->N == 0) return ROCS_OK;
+  DcaItemList items;
+  rocs_status_t st = plan_dca_items(plan, BQ / n_q, H, stream, &items);
+  if (st != ROCS_OK) return st;
+  if (items.num == 0) return ROCS_OK;
+  const uint64_t width = (uint64_t)H * DH;
+  CUtensorMap map_q, map_k, map_v;
+  if (!make_tensor_map_2d(&map_q, Q, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, (uint64_t)plan->N * n_q, width, width, BQ, DH,
+                          true))
+    return ROCS_ERR_CUDA;
+  if (T > 0) {
+    if (!make_tensor_map_2d(&map_k, K, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, (uint64_t)T, width, width, BKV, DH, true) ||
+        !make_tensor_map_2d(&map_v, V, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, (uint64_t)T, width, width, BKV, DH, true))
+      return ROCS_ERR_CUDA;
+  } else {
+    map_k = map_q;  // every sequence is empty: the kernel only writes zeros
+    map_v = map_q;
+  }
+  uint32_t* status = device_status_word();
+  if (!status) return ROCS_ERR_CUDA;
+  DcaParams p{};
+  p.items = items.dev;
+  p.num_items = items.num;
+  p.n_q = n_q;
+  p.H = H;
+  p.scale_log2e = scale * 1.4426950408889634f;
+  p.seq_offsets = seq_offsets;
+  p.O = (__nv_bfloat16*)O;
+  p.n_rows = plan->N * n_q;
+  p.status = status;
+  ROCS_CUDA_TRY(cudaFuncSetAttribute(dca_umma_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes));
+  const int grid = std::min(items.num, sm_count_dca());
+  dca_umma_kernel<<<grid, kThreads, kSmemBytes, stream>>>(map_q, map_k, map_v, p);
+  ROCS_CUDA_TRY(cudaGetLastError());
+  return ROCS_OK;
+}
+
+}  // namespace rocs

@@ -188,52 +188,47 @@ glm_umma_kernel(const __grid_constant__ CUtensorMap map_xr, const __grid_constan
       if (!mbar_wait(&tmem_full[g], (it >> 1) & 1, abort_flag, p.status, kStatusGlm | 4)) break;
       tc_fence_after_sync();
       const uint32_t t_row = tmem_base + g * kAccStride + ((uint32_t)(q * 32) << 16);
-      // request-candidate block: columns 0 .. n_r-1 (n_r is a multiple of 8)
-      for (int32_t c0 = 0; c0 < p.n_r; c0 += 16) {
-        uint32_t v[16];
-        tmem_ld_32x32b_x16(t_row + c0, v);
+      // All TMEM reads of the tile are issued before the first wait: the first 32 columns of the
+      // request-candidate block and the 32 x 32 diagonal block of this warp's rows.
+      uint32_t vcr[32], vcc[32];
+      tmem_ld_32x32b_x32(t_row, vcr);
+      tmem_ld_32x32b_x32(t_row + p.n_r_pad + q * 32, vcc);
+      tmem_ld_wait();
+      auto store8 = [&](const uint32_t* v, int32_t col) {
+        uint4 w;
+        __nv_bfloat162 b2;
+        b2 = __floats2bfloat162_rn(__uint_as_float(v[0]), __uint_as_float(v[1])); w.x = *reinterpret_cast<uint32_t*>(&b2);
+        b2 = __floats2bfloat162_rn(__uint_as_float(v[2]), __uint_as_float(v[3])); w.y = *reinterpret_cast<uint32_t*>(&b2);
+        b2 = __floats2bfloat162_rn(__uint_as_float(v[4]), __uint_as_float(v[5])); w.z = *reinterpret_cast<uint32_t*>(&b2);
+        b2 = __floats2bfloat162_rn(__uint_as_float(v[6]), __uint_as_float(v[7])); w.w = *reinterpret_cast<uint32_t*>(&b2);
+        *reinterpret_cast<uint4*>(my + col * 2) = w;
+      };
+#pragma unroll
+      for (int h = 0; h < 4; ++h)
+        if (8 * h < p.n_r) store8(vcr + 8 * h, 8 * h);
+      for (int32_t c0 = 32; c0 < p.n_r; c0 += 32) {  // wider request blocks: 32 more columns per pass
+        tmem_ld_32x32b_x32(t_row + c0, vcr);
         tmem_ld_wait();
 #pragma unroll
-        for (int h = 0; h < 2; ++h) {
-          if (c0 + 8 * h < p.n_r) {
-            uint4 w;
-            __nv_bfloat162 b2;
-            b2 = __floats2bfloat162_rn(__uint_as_float(v[8 * h + 0]), __uint_as_float(v[8 * h + 1])); w.x = *reinterpret_cast<uint32_t*>(&b2);
-            b2 = __floats2bfloat162_rn(__uint_as_float(v[8 * h + 2]), __uint_as_float(v[8 * h + 3])); w.y = *reinterpret_cast<uint32_t*>(&b2);
-            b2 = __floats2bfloat162_rn(__uint_as_float(v[8 * h + 4]), __uint_as_float(v[8 * h + 5])); w.z = *reinterpret_cast<uint32_t*>(&b2);
-            b2 = __floats2bfloat162_rn(__uint_as_float(v[8 * h + 6]), __uint_as_float(v[8 * h + 7])); w.w = *reinterpret_cast<uint32_t*>(&b2);
-            *reinterpret_cast<uint4*>(my + (c0 + 8 * h) * 2) = w;
-          }
-        }
+        for (int h = 0; h < 4; ++h)
+          if (c0 + 8 * h < p.n_r) store8(vcr + 8 * h, c0 + 8 * h);
       }
-      // candidate-candidate block: the 32 x 32 diagonal block of this warp's rows, of which each
-      // thread keeps the NC columns of its own candidate
+      tc_fence_before_sync();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(&tmem_empty[g]);
       {
-        uint32_t v[32];
-        tmem_ld_32x32b_x32(t_row + p.n_r_pad + q * 32, v);
-        tmem_ld_wait();
-        tc_fence_before_sync();
-        __syncwarp();
-        if (lane == 0) mbar_arrive(&tmem_empty[g]);
-        const int sub = lane / NC;  // which candidate of the warp's 32 / NC this row belongs to
-        float x[NC];
+        // of the diagonal block each thread keeps the NC columns of its own candidate
+        const int sub = lane / NC;
+        uint32_t x[NC];
 #pragma unroll
         for (int j = 0; j < NC; ++j) {
-          uint32_t xv = v[j];
+          uint32_t xv = vcc[j];
 #pragma unroll
-          for (int s2 = 1; s2 < 32 / NC; ++s2) xv = (sub == s2) ? v[s2 * NC + j] : xv;
-          x[j] = __uint_as_float(xv);
+          for (int s2 = 1; s2 < 32 / NC; ++s2) xv = (sub == s2) ? vcc[s2 * NC + j] : xv;
+          x[j] = xv;
         }
 #pragma unroll
-        for (int j = 0; j < NC; j += 8) {
-          uint4 w;
-          __nv_bfloat162 b2;
-          b2 = __floats2bfloat162_rn(x[j + 0], x[j + 1]); w.x = *reinterpret_cast<uint32_t*>(&b2);
-          b2 = __floats2bfloat162_rn(x[j + 2], x[j + 3]); w.y = *reinterpret_cast<uint32_t*>(&b2);
-          b2 = __floats2bfloat162_rn(x[j + 4], x[j + 5]); w.z = *reinterpret_cast<uint32_t*>(&b2);
-          b2 = __floats2bfloat162_rn(x[j + 6], x[j + 7]); w.w = *reinterpret_cast<uint32_t*>(&b2);
-          *reinterpret_cast<uint4*>(my + (p.n_r + j) * 2) = w;
-        }
+        for (int j = 0; j < NC; j += 8) store8(x + j, p.n_r + j);
       }
       __syncwarp();
       const int32_t rows_valid = min(32, tile.count * NC - q * 32);  // this warp's rows that are real
@@ -254,40 +249,52 @@ glm_umma_kernel(const __grid_constant__ CUtensorMap map_xr, const __grid_constan
         const int32_t cands = rows_valid / NC;
         for (int32_t cl = 0; cl < cands; ++cl) {
           __nv_bfloat16* oc = p.OC + ((int64_t)tile.cand0 + q * (32 / NC) + cl) * p.n_co * n;
-          for (int32_t j = 0; j < n8; ++j) {
-            float d0 = 0.f, d1 = 0.f, d2 = 0.f, d3 = 0.f;
-            const int32_t col = 8 * j + 2 * t4;
-            if (g8 < p.n_co) {
-              const float2 z = __ldg(reinterpret_cast<const float2*>(zr + g8 * n + col));
-              d0 = z.x; d1 = z.y;
-            }
-            if (g8 + 8 < p.n_co) {
-              const float2 z = __ldg(reinterpret_cast<const float2*>(zr + (g8 + 8) * n + col));
-              d2 = z.x; d3 = z.y;
+          // six 8-column blocks at a time, all loads first, so the tensor-core ops overlap
+          for (int32_t j0 = 0; j0 < n8; j0 += 6) {
+            float dd[6][4];
+            uint32_t bb[6][KS][2];
+#pragma unroll
+            for (int u = 0; u < 6; ++u) {
+              const int32_t j = min(j0 + u, n8 - 1);
+              const int32_t col = 8 * j + 2 * t4;
+              dd[u][0] = dd[u][1] = dd[u][2] = dd[u][3] = 0.f;
+              if (g8 < p.n_co) {
+                const float2 z = __ldg(reinterpret_cast<const float2*>(zr + g8 * n + col));
+                dd[u][0] = z.x; dd[u][1] = z.y;
+              }
+              if (g8 + 8 < p.n_co) {
+                const float2 z = __ldg(reinterpret_cast<const float2*>(zr + (g8 + 8) * n + col));
+                dd[u][2] = z.x; dd[u][3] = z.y;
+              }
+#pragma unroll
+              for (int ks = 0; ks < KS; ++ks) {
+                bb[u][ks][1] = 0u;
+                if constexpr (NC >= 16) {
+                  const uint32_t addr = smem_u32(yc_w + (cl * NC + ks * 16 + (lane & 15)) * p.yc_stride + j * 16);
+                  asm volatile("ldmatrix.sync.aligned.m8n8.x2.trans.shared.b16 {%0, %1}, [%2];"
+                               : "=r"(bb[u][ks][0]), "=r"(bb[u][ks][1]) : "r"(addr));
+                } else {
+                  const uint32_t addr8 = smem_u32(yc_w + (cl * NC + (lane & 7)) * p.yc_stride + j * 16);
+                  asm volatile("ldmatrix.sync.aligned.m8n8.x1.trans.shared.b16 {%0}, [%1];" : "=r"(bb[u][ks][0]) : "r"(addr8));
+                }
+              }
             }
 #pragma unroll
-            for (int ks = 0; ks < KS; ++ks) {
-              uint32_t b0, b1 = 0u;
-              const uint32_t addr = smem_u32(yc_w + (cl * NC + ks * 16 + (lane & 15)) * p.yc_stride + j * 16);
-              if constexpr (NC >= 16) {
-                asm volatile("ldmatrix.sync.aligned.m8n8.x2.trans.shared.b16 {%0, %1}, [%2];" : "=r"(b0), "=r"(b1) : "r"(addr));
-              } else {
-                const uint32_t addr8 = smem_u32(yc_w + (cl * NC + (lane & 7)) * p.yc_stride + j * 16);
-                asm volatile("ldmatrix.sync.aligned.m8n8.x1.trans.shared.b16 {%0}, [%1];" : "=r"(b0) : "r"(addr8));
-              }
-              asm volatile(
-                  "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0, %1, %2, %3}, {%4, %5, %6, %7}, {%8, %9}, "
-                  "{%0, %1, %2, %3};"
-                  : "+f"(d0), "+f"(d1), "+f"(d2), "+f"(d3)
-                  : "r"(wa[ks][0]), "r"(wa[ks][1]), "r"(wa[ks][2]), "r"(wa[ks][3]), "r"(b0), "r"(b1));
-            }
-            if (g8 < p.n_co) {
-              __nv_bfloat162 h2 = __floats2bfloat162_rn(d0, d1);
-              *reinterpret_cast<__nv_bfloat162*>(oc + g8 * n + col) = h2;
-            }
-            if (g8 + 8 < p.n_co) {
-              __nv_bfloat162 h2 = __floats2bfloat162_rn(d2, d3);
-              *reinterpret_cast<__nv_bfloat162*>(oc + (g8 + 8) * n + col) = h2;
+            for (int u = 0; u < 6; ++u)
+#pragma unroll
+              for (int ks = 0; ks < KS; ++ks)
+                asm volatile(
+                    "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0, %1, %2, %3}, {%4, %5, %6, %7}, {%8, %9}, "
+                    "{%0, %1, %2, %3};"
+                    : "+f"(dd[u][0]), "+f"(dd[u][1]), "+f"(dd[u][2]), "+f"(dd[u][3])
+                    : "r"(wa[ks][0]), "r"(wa[ks][1]), "r"(wa[ks][2]), "r"(wa[ks][3]), "r"(bb[u][ks][0]), "r"(bb[u][ks][1]));
+#pragma unroll
+            for (int u = 0; u < 6; ++u) {
+              if (j0 + u >= n8) continue;
+              const int32_t col = 8 * (j0 + u) + 2 * t4;
+              if (g8 < p.n_co) *reinterpret_cast<__nv_bfloat162*>(oc + g8 * n + col) = __floats2bfloat162_rn(dd[u][0], dd[u][1]);
+              if (g8 + 8 < p.n_co)
+                *reinterpret_cast<__nv_bfloat162*>(oc + (g8 + 8) * n + col) = __floats2bfloat162_rn(dd[u][2], dd[u][3]);
             }
           }
         }
