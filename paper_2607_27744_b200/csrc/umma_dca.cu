@@ -10,11 +10,16 @@
 //   warp 0     TMA producer: Q tiles of the item, then (K_j, V_j) blocks through a ring
 //   warp 1     tcgen05.mma issuer:  S_X = Q_X K_j^T  (128x128x64)  and  O_X = P_X V_j  (128x64x128)
 //   warps 2-5  softmax group A,  warps 6-9  softmax group B: each thread owns one query row:
-//              TMEM -> registers, running max and sum in fp32 (exp2 on scaled scores), P rounded to
-//              bf16 into shared memory (the A operand of the second MMA), O accumulated in registers
-//              across key blocks (O = O * alpha + P V), final 1/sum, bf16 store.
-// The two groups run half a phase apart, so while one waits for its next S tile the other keeps the
-// exponential unit busy.  Every row's arithmetic depends only on that row and its request's K/V.
+//              S from TMEM into registers (one read), reference max and sum in fp32 (exp2 on scaled
+//              scores), P rounded to bf16 into shared memory (the A operand of the second MMA),
+//              final 1/sum, bf16 store.
+// O accumulates in TMEM across key blocks.  A row moves its reference max only when the block max
+// exceeds it by more than 2^8; then O is rescaled in TMEM (read, multiply, write back) before the
+// next P V is issued.  The decision is taken per row from that row's own scores; rows that keep
+// their reference multiply by exactly 1, so a row's bits never depend on its neighbours.
+// Q is double buffered and the producer runs one item ahead, so consecutive items overlap; the two
+// groups run out of phase, so while one waits for its next S tile the other keeps the exponential
+// unit busy.
 #include <algorithm>
 
 #include "rocs_internal.h"
@@ -33,7 +38,8 @@ constexpr int kKvStages = 3;
 constexpr int kQBytes = BQ * DH * 2;          // 16 KB
 constexpr int kKvStageBytes = 2 * BKV * DH * 2;  // K block + V block = 32 KB
 constexpr int kPBytes = BQ * BKV * 2;         // 32 KB per side
-constexpr int kSmemBytes = 2 * kQBytes + kKvStages * kKvStageBytes + 2 * kPBytes + 256 + 1024;
+constexpr int kSmemBytes = 4 * kQBytes + kKvStages * kKvStageBytes + 2 * kPBytes + 512 + 1024;
+constexpr float kRescaleThreshold = 8.f;  // log2 units
 constexpr uint32_t kStatusDca = 0x400;
 constexpr int kSideTmemStride = 256;  // side A: columns 0.., side B: columns 256..
 constexpr int kOColOffset = 128;      // S in [0, 128), O block in [128, 192) of the side
@@ -60,16 +66,16 @@ dca_umma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
                 const __grid_constant__ CUtensorMap map_v, const DcaParams p) {
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
-  uint8_t* q_smem = smem;                              // [2][128][64] bf16
-  uint8_t* kv_smem = q_smem + 2 * kQBytes;             // [stages][K 16 KB | V 16 KB]
+  uint8_t* q_smem = smem;                              // [2 slots][2 sides][128][64] bf16
+  uint8_t* kv_smem = q_smem + 4 * kQBytes;             // [stages][K 16 KB | V 16 KB]
   uint8_t* p_smem = kv_smem + kKvStages * kKvStageBytes;  // [2][2 x (128 x 64)] bf16, K-major swizzled
-  uint64_t* q_full = reinterpret_cast<uint64_t*>(p_smem + 2 * kPBytes);
-  uint64_t* item_done = q_full + 1;
-  uint64_t* item_start = item_done + 1;
-  uint64_t* kv_full = item_start + 1;
+  uint64_t* q_full = reinterpret_cast<uint64_t*>(p_smem + 2 * kPBytes);  // [2]
+  uint64_t* q_empty = q_full + 2;            // [2]
+  uint64_t* kv_full = q_empty + 2;
   uint64_t* kv_empty = kv_full + kKvStages;
   uint64_t* s_full = kv_empty + kKvStages;   // [2]
-  uint64_t* p_full = s_full + 2;             // [2]
+  uint64_t* s_empty = s_full + 2;            // [2]
+  uint64_t* p_full = s_empty + 2;            // [2]
   uint64_t* o_full = p_full + 2;             // [2]
   uint64_t* drain = o_full + 2;
   uint32_t* tmem_ptr = reinterpret_cast<uint32_t*>(drain + 1);
@@ -78,15 +84,17 @@ dca_umma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
   const int warp = threadIdx.x / 32, lane = threadIdx.x % 32;
 
   if (threadIdx.x == 0) {
-    mbar_init(q_full, 1);
-    mbar_init(item_done, 8);
-    mbar_init(item_start, 1);
+    for (int x = 0; x < 2; ++x) {
+      mbar_init(&q_full[x], 1);
+      mbar_init(&q_empty[x], 1);
+    }
     for (int s = 0; s < kKvStages; ++s) {
       mbar_init(&kv_full[s], 1);
       mbar_init(&kv_empty[s], 1);
     }
     for (int x = 0; x < 2; ++x) {
       mbar_init(&s_full[x], 1);
+      mbar_init(&s_empty[x], 4);
       mbar_init(&p_full[x], 4);
       mbar_init(&o_full[x], 1);
     }
@@ -110,20 +118,21 @@ dca_umma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
       prefetch_tensormap(&map_q);
       prefetch_tensormap(&map_k);
       prefetch_tensormap(&map_v);
-      uint32_t kv_it = 0, n_item = 0;
+      uint32_t kv_it = 0, n_work = 0;
       bool ok = true;
-      for (int32_t i = blockIdx.x; i < p.num_items && ok; i += gridDim.x, ++n_item) {
+      for (int32_t i = blockIdx.x; i < p.num_items && ok; i += gridDim.x) {
         const DcaItem item = p.items[i];
         const int32_t s0 = p.seq_offsets[item.req];
         const int32_t L = p.seq_offsets[item.req + 1] - s0;
-        // Q buffers are free once both softmax groups have finished the previous item
-        if (!mbar_wait(item_done, (n_item & 1) ^ 1, abort_flag, p.status, kStatusDca | 1)) { ok = false; break; }
-        mbar_arrive(item_start);  // the softmax warps may enter this item (keeps them in step, also when idle)
-        if (L == 0) continue;
+        if (L == 0) continue;  // nobody touches a barrier for an item without keys
+        const uint32_t slot = n_work & 1;
+        if (!mbar_wait(&q_empty[slot], ((n_work >> 1) & 1) ^ 1, abort_flag, p.status, kStatusDca | 1)) { ok = false; break; }
+        ++n_work;
         const int32_t sides = item.count_b > 0 ? 2 : 1;
-        mbar_expect_tx(q_full, sides * kQBytes);
-        tma_load_2d(q_smem, &map_q, q_full, item.head * DH, item.cand0 * p.n_q);
-        if (sides == 2) tma_load_2d(q_smem + kQBytes, &map_q, q_full, item.head * DH, (item.cand0 + item.count_a) * p.n_q);
+        uint8_t* qs = q_smem + slot * 2 * kQBytes;
+        mbar_expect_tx(&q_full[slot], sides * kQBytes);
+        tma_load_2d(qs, &map_q, &q_full[slot], item.head * DH, item.cand0 * p.n_q);
+        if (sides == 2) tma_load_2d(qs + kQBytes, &map_q, &q_full[slot], item.head * DH, (item.cand0 + item.count_a) * p.n_q);
         const int32_t nblk = (L + BKV - 1) / BKV;
         for (int32_t j = 0; j < nblk; ++j, ++kv_it) {
           const int s = kv_it % kKvStages;
@@ -150,15 +159,16 @@ dca_umma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
     uint32_t kv_it = 0, n_work = 0;           // n_work: items that had keys (phase of q_full)
     uint32_t cnt_p[2] = {0, 0};               // phases of p_full per side
     bool ok = true;
-    auto issue_s = [&](int side, int stage) {
+    uint32_t cnt_se[2] = {0, 0};              // phases of s_empty per side
+    auto issue_s = [&](int side, int stage, uint32_t slot) {
       const uint32_t d = tmem_base + side * kSideTmemStride;
-      const uint64_t a_desc = smem_desc_sw128(smem_u32(q_smem + side * kQBytes), 1024, 16);
+      const uint64_t a_desc = smem_desc_sw128(smem_u32(q_smem + (slot * 2 + side) * kQBytes), 1024, 16);
       const uint64_t b_desc = smem_desc_sw128(smem_u32(kv_smem + stage * kKvStageBytes), 1024, 16);
 #pragma unroll
       for (int k = 0; k < DH / 16; ++k) umma_ss(d, a_desc + 2 * k, b_desc + 2 * k, idesc_s, k != 0 ? 1u : 0u);
       umma_commit(&s_full[side]);
     };
-    auto issue_pv = [&](int side, int stage) {
+    auto issue_pv = [&](int side, int stage, bool first_block) {
       const uint32_t d = tmem_base + side * kSideTmemStride + kOColOffset;
       const uint32_t p_addr = smem_u32(p_smem + side * kPBytes);
       const uint32_t v_addr = smem_u32(kv_smem + stage * kKvStageBytes + BKV * DH * 2);
@@ -168,7 +178,7 @@ dca_umma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
         const uint64_t a_desc = smem_desc_sw128(p_addr + (k / 4) * (BQ * 128) + (k % 4) * 32, 1024, 16);
         // V: rows are keys (K), 128 bytes = 64 head dims (N): 16 keys = 2048 bytes further on
         const uint64_t b_desc = smem_desc_sw128(v_addr + k * 16 * 128, 1024, 16);
-        umma_ss(d, a_desc, b_desc, idesc_o, k != 0 ? 1u : 0u);
+        umma_ss(d, a_desc, b_desc, idesc_o, (k != 0 || !first_block) ? 1u : 0u);
       }
       umma_commit(&o_full[side]);
     };
@@ -178,29 +188,47 @@ dca_umma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
       if (L == 0) continue;
       const int32_t sides = item.count_b > 0 ? 2 : 1;
       const int32_t nblk = (L + BKV - 1) / BKV;
-      if (!mbar_wait(q_full, n_work & 1, abort_flag, p.status, kStatusDca | 3)) { ok = false; break; }
+      const uint32_t slot = n_work & 1;
+      if (!mbar_wait(&q_full[slot], (n_work >> 1) & 1, abort_flag, p.status, kStatusDca | 3)) { ok = false; break; }
       ++n_work;
-      // first key block: S for both sides
+      // first key block: S for both sides (their S tiles were drained at the end of the previous item)
       if (!mbar_wait(&kv_full[kv_it % kKvStages], (kv_it / kKvStages) & 1, abort_flag, p.status, kStatusDca | 4)) { ok = false; break; }
       tc_fence_after_sync();
-      if (lane == 0)
-        for (int x = 0; x < sides; ++x) issue_s(x, kv_it % kKvStages);
+      if (lane == 0) {
+        for (int x = 0; x < sides; ++x) issue_s(x, kv_it % kKvStages, slot);
+        if (nblk == 1) umma_commit(&q_empty[slot]);
+      }
       __syncwarp();
       for (int32_t j = 0; j < nblk && ok; ++j, ++kv_it) {
         const int stage = kv_it % kKvStages;
         const int next_stage = (kv_it + 1) % kKvStages;
         if (j + 1 < nblk) {
           if (!mbar_wait(&kv_full[next_stage], ((kv_it + 1) / kKvStages) & 1, abort_flag, p.status, kStatusDca | 5)) { ok = false; break; }
+          // S_{j+1} as soon as the side has pulled S_j into registers
+          for (int x = 0; x < sides; ++x) {
+            if (!mbar_wait(&s_empty[x], cnt_se[x] & 1, abort_flag, p.status, kStatusDca | 11)) { ok = false; break; }
+            ++cnt_se[x];
+            tc_fence_after_sync();
+            if (lane == 0) issue_s(x, next_stage, slot);
+            __syncwarp();
+          }
+          if (!ok) break;
+          if (j + 2 == nblk && lane == 0) umma_commit(&q_empty[slot]);  // last S of the item: Q slot is free
+          __syncwarp();
+        } else {
+          // keep the s_empty phases in step: the sides still signal after reading the last S
+          for (int x = 0; x < sides; ++x) {
+            if (!mbar_wait(&s_empty[x], cnt_se[x] & 1, abort_flag, p.status, kStatusDca | 12)) { ok = false; break; }
+            ++cnt_se[x];
+          }
+          if (!ok) break;
         }
         for (int x = 0; x < sides; ++x) {
-          // P_j of this side is in shared memory and its S tile has been read
+          // P_j of this side is in shared memory (and O has been rescaled if it had to be)
           if (!mbar_wait(&p_full[x], cnt_p[x] & 1, abort_flag, p.status, kStatusDca | 6)) { ok = false; break; }
           ++cnt_p[x];
           tc_fence_after_sync();
-          if (lane == 0) {
-            issue_pv(x, stage);
-            if (j + 1 < nblk) issue_s(x, next_stage);
-          }
+          if (lane == 0) issue_pv(x, stage, j == 0);
           __syncwarp();
         }
         if (ok && lane == 0) umma_commit(&kv_empty[stage]);  // K_j and V_j are no longer needed
@@ -220,9 +248,8 @@ dca_umma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
     const uint32_t t_s = tmem_base + side * kSideTmemStride + ((uint32_t)(q * 32) << 16);
     const uint32_t t_o = t_s + kOColOffset;
     uint8_t* p_row = p_smem + side * kPBytes + row * 128;
-    uint32_t cnt_s = 0, cnt_o = 0, n_item = 0;
-    for (int32_t i = blockIdx.x; i < p.num_items; i += gridDim.x, ++n_item) {
-      if (!mbar_wait(item_start, n_item & 1, abort_flag, p.status, kStatusDca | 10)) break;
+    uint32_t cnt_s = 0, cnt_o = 0;
+    for (int32_t i = blockIdx.x; i < p.num_items; i += gridDim.x) {
       const DcaItem item = p.items[i];
       const int32_t L = p.seq_offsets[item.req + 1] - p.seq_offsets[item.req];
       const int32_t my_count = side == 0 ? item.count_a : item.count_b;
@@ -233,7 +260,7 @@ dca_umma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
       float o_reg[DH];
 #pragma unroll
       for (int e = 0; e < DH; ++e) o_reg[e] = 0.f;
-      float m_run = -INFINITY, l_run = 0.f, alpha_pending = 0.f;
+      float m_ref = -INFINITY, l_run = 0.f;
       if (my_count > 0 && L > 0) {
         const int32_t nblk = (L + BKV - 1) / BKV;
         for (int32_t j = 0; j < nblk; ++j) {
@@ -241,64 +268,60 @@ dca_umma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
           if (!mbar_wait(&s_full[side], cnt_s & 1, abort_flag, p.status, kStatusDca | 7)) { aborted = true; break; }
           ++cnt_s;
           tc_fence_after_sync();
-          // pass 1: row maximum of the scaled scores
-          float mx = -INFINITY;
-#pragma unroll 1
-          for (int c = 0; c < BKV; c += 32) {
-            uint32_t v[32];
-            tmem_ld_32x32b_x32(t_s + c, v);
-            tmem_ld_wait();
+          uint32_t sv[BKV];
 #pragma unroll
-            for (int e = 0; e < 32; ++e) {
-              const float s = __uint_as_float(v[e]) * p.scale_log2e;
-              mx = fmaxf(mx, (c + e < valid) ? s : -INFINITY);
-            }
+          for (int c = 0; c < BKV; c += 32) tmem_ld_32x32b_x32(t_s + c, sv + c);
+          tmem_ld_wait();
+          tc_fence_before_sync();
+          __syncwarp();
+          if (lane == 0) mbar_arrive(&s_empty[side]);  // S_{j+1} may overwrite the tile now
+          if (valid < BKV) {
+#pragma unroll
+            for (int e = 0; e < BKV; ++e)
+              if (e >= valid) sv[e] = 0xff800000u;  // -inf: the key does not exist
           }
-          const float m_new = fmaxf(m_run, mx);
-          const float alpha = ex2(m_run - m_new);  // 0 for the first block (m_run = -inf)
-          // fold the previous block's P V into the running output; this also tells us that the MMA
-          // has finished reading the previous P from shared memory
+          float mx = -INFINITY;
+#pragma unroll
+          for (int e = 0; e < BKV; ++e) mx = fmaxf(mx, __uint_as_float(sv[e]));
+          mx *= p.scale_log2e;
+          // this row's own decision: move the reference only for a jump of more than 2^8
+          const bool move = mx > m_ref + kRescaleThreshold;
+          const float m_new = move ? mx : m_ref;
+          const float alpha = move ? ex2(m_ref - m_new) : 1.f;  // 0 on the first block
+          m_ref = m_new;
           if (j > 0) {
+            // P V of the previous block is complete: O is stable and P's buffer may be rewritten
             if (!mbar_wait(&o_full[side], cnt_o & 1, abort_flag, p.status, kStatusDca | 8)) { aborted = true; break; }
             ++cnt_o;
             tc_fence_after_sync();
+            if (__any_sync(0xffffffffu, move)) {
 #pragma unroll
-            for (int c = 0; c < DH; c += 32) {
-              uint32_t v[32];
-              tmem_ld_32x32b_x32(t_o + c, v);
-              tmem_ld_wait();
+              for (int c = 0; c < DH; c += 16) {
+                uint32_t v[16];
+                tmem_ld_32x32b_x16(t_o + c, v);
+                tmem_ld_wait();
 #pragma unroll
-              for (int e = 0; e < 32; ++e) o_reg[c + e] = fmaf(o_reg[c + e], alpha_pending, __uint_as_float(v[e]));
+                for (int e = 0; e < 16; ++e) v[e] = __float_as_uint(__uint_as_float(v[e]) * alpha);
+                tmem_st_32x32b_x16(t_o + c, v);
+              }
+              tmem_st_wait();
             }
           }
-          alpha_pending = alpha;
-          m_run = m_new;
-          // pass 2: P = exp2(s - m), row sum, bf16 P into the swizzled K-major operand layout
           float sum = 0.f;
-#pragma unroll 1
-          for (int c = 0; c < BKV; c += 32) {
-            uint32_t v[32];
-            tmem_ld_32x32b_x32(t_s + c, v);
-            tmem_ld_wait();
-            uint32_t packed[16];
 #pragma unroll
-            for (int e = 0; e < 32; e += 2) {
-              float p0 = ex2(fmaf(__uint_as_float(v[e]), p.scale_log2e, -m_new));
-              float p1 = ex2(fmaf(__uint_as_float(v[e + 1]), p.scale_log2e, -m_new));
-              p0 = (c + e < valid) ? p0 : 0.f;
-              p1 = (c + e + 1 < valid) ? p1 : 0.f;
-              sum += p0 + p1;
-              __nv_bfloat162 h2 = __floats2bfloat162_rn(p0, p1);
-              packed[e / 2] = *reinterpret_cast<uint32_t*>(&h2);
-            }
-            // 32 keys = four 16-byte chunks of this row inside the 64-key block c / 64
-            uint8_t* blk = p_row + (c / 64) * (BQ * 128);
+          for (int c = 0; c < BKV; c += 8) {
+            float pe[8];
 #pragma unroll
-            for (int u = 0; u < 4; ++u) {
-              const int chunk = (c % 64) / 8 + u;
-              *reinterpret_cast<uint4*>(blk + ((chunk ^ (row & 7)) << 4)) =
-                  make_uint4(packed[4 * u], packed[4 * u + 1], packed[4 * u + 2], packed[4 * u + 3]);
-            }
+            for (int e = 0; e < 8; ++e) pe[e] = ex2(fmaf(__uint_as_float(sv[c + e]), p.scale_log2e, -m_new));
+            sum += ((pe[0] + pe[1]) + (pe[2] + pe[3])) + ((pe[4] + pe[5]) + (pe[6] + pe[7]));
+            uint4 w;
+            __nv_bfloat162 h2;
+            h2 = __floats2bfloat162_rn(pe[0], pe[1]); w.x = *reinterpret_cast<uint32_t*>(&h2);
+            h2 = __floats2bfloat162_rn(pe[2], pe[3]); w.y = *reinterpret_cast<uint32_t*>(&h2);
+            h2 = __floats2bfloat162_rn(pe[4], pe[5]); w.z = *reinterpret_cast<uint32_t*>(&h2);
+            h2 = __floats2bfloat162_rn(pe[6], pe[7]); w.w = *reinterpret_cast<uint32_t*>(&h2);
+            // 8 keys = one 16-byte chunk of this row inside the 64-key block c / 64
+            *reinterpret_cast<uint4*>(p_row + (c / 64) * (BQ * 128) + ((((c % 64) / 8) ^ (row & 7)) << 4)) = w;
           }
           l_run = l_run * alpha + sum;
           fence_proxy_async_smem();
@@ -318,7 +341,7 @@ dca_umma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
               tmem_ld_32x32b_x32(t_o + c, v);
               tmem_ld_wait();
 #pragma unroll
-              for (int e = 0; e < 32; ++e) o_reg[c + e] = fmaf(o_reg[c + e], alpha_pending, __uint_as_float(v[e]));
+              for (int e = 0; e < 32; ++e) o_reg[c + e] = __uint_as_float(v[e]);
             }
           }
         }
@@ -337,9 +360,7 @@ dca_umma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
           *reinterpret_cast<uint4*>(out + c) = w;
         }
       }
-      tc_fence_before_sync();
-      __syncwarp();
-      if (lane == 0) mbar_arrive(item_done);
+      tc_fence_before_sync();  // the next item's first P V overwrites O
     }
   }
 
