@@ -257,9 +257,6 @@ dca_umma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
       const int32_t rows_valid = my_count * p.n_q;
       __nv_bfloat16* out = p.O + ((int64_t)cand_first * p.n_q + row) * row_width + item.head * DH;
       bool aborted = false;
-      float o_reg[DH];
-#pragma unroll
-      for (int e = 0; e < DH; ++e) o_reg[e] = 0.f;
       float m_ref = -INFINITY, l_run = 0.f;
       if (my_count > 0 && L > 0) {
         const int32_t nblk = (L + BKV - 1) / BKV;
@@ -280,9 +277,13 @@ dca_umma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
             for (int e = 0; e < BKV; ++e)
               if (e >= valid) sv[e] = 0xff800000u;  // -inf: the key does not exist
           }
-          float mx = -INFINITY;
+          float mx4[8];
 #pragma unroll
-          for (int e = 0; e < BKV; ++e) mx = fmaxf(mx, __uint_as_float(sv[e]));
+          for (int u = 0; u < 8; ++u) mx4[u] = __uint_as_float(sv[u]);
+#pragma unroll
+          for (int e = 8; e < BKV; ++e) mx4[e & 7] = fmaxf(mx4[e & 7], __uint_as_float(sv[e]));  // 8 short chains
+          float mx = fmaxf(fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3])),
+                           fmaxf(fmaxf(mx4[4], mx4[5]), fmaxf(mx4[6], mx4[7])));
           mx *= p.scale_log2e;
           // this row's own decision: move the reference only for a jump of more than 2^8
           const bool move = mx > m_ref + kRescaleThreshold;
@@ -335,31 +336,33 @@ dca_umma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
           } else {
             ++cnt_o;
             tc_fence_after_sync();
+            const float inv = 1.f / l_run;
 #pragma unroll
             for (int c = 0; c < DH; c += 32) {
               uint32_t v[32];
               tmem_ld_32x32b_x32(t_o + c, v);
               tmem_ld_wait();
+              if (row < rows_valid) {
 #pragma unroll
-              for (int e = 0; e < 32; ++e) o_reg[c + e] = __uint_as_float(v[e]);
+                for (int e = 0; e < 32; e += 8) {
+                  uint4 w;
+                  __nv_bfloat162 h2;
+                  h2 = __floats2bfloat162_rn(__uint_as_float(v[e + 0]) * inv, __uint_as_float(v[e + 1]) * inv); w.x = *reinterpret_cast<uint32_t*>(&h2);
+                  h2 = __floats2bfloat162_rn(__uint_as_float(v[e + 2]) * inv, __uint_as_float(v[e + 3]) * inv); w.y = *reinterpret_cast<uint32_t*>(&h2);
+                  h2 = __floats2bfloat162_rn(__uint_as_float(v[e + 4]) * inv, __uint_as_float(v[e + 5]) * inv); w.z = *reinterpret_cast<uint32_t*>(&h2);
+                  h2 = __floats2bfloat162_rn(__uint_as_float(v[e + 6]) * inv, __uint_as_float(v[e + 7]) * inv); w.w = *reinterpret_cast<uint32_t*>(&h2);
+                  *reinterpret_cast<uint4*>(out + c + e) = w;
+                }
+              }
             }
           }
         }
+      } else if (my_count > 0 && row < rows_valid) {
+        // a request without keys: zero rows
+#pragma unroll
+        for (int c = 0; c < DH; c += 8) *reinterpret_cast<uint4*>(out + c) = make_uint4(0u, 0u, 0u, 0u);
       }
       if (aborted) break;
-      if (row < rows_valid) {
-        const float inv = (L > 0) ? 1.f / l_run : 0.f;
-#pragma unroll
-        for (int c = 0; c < DH; c += 8) {
-          uint4 w;
-          __nv_bfloat162 h2;
-          h2 = __floats2bfloat162_rn(o_reg[c + 0] * inv, o_reg[c + 1] * inv); w.x = *reinterpret_cast<uint32_t*>(&h2);
-          h2 = __floats2bfloat162_rn(o_reg[c + 2] * inv, o_reg[c + 3] * inv); w.y = *reinterpret_cast<uint32_t*>(&h2);
-          h2 = __floats2bfloat162_rn(o_reg[c + 4] * inv, o_reg[c + 5] * inv); w.z = *reinterpret_cast<uint32_t*>(&h2);
-          h2 = __floats2bfloat162_rn(o_reg[c + 6] * inv, o_reg[c + 7] * inv); w.w = *reinterpret_cast<uint32_t*>(&h2);
-          *reinterpret_cast<uint4*>(out + c) = w;
-        }
-      }
       tc_fence_before_sync();  // the next item's first P V overwrites O
     }
   }
