@@ -165,20 +165,26 @@ __global__ void __launch_bounds__(DCA_WARPS * 32) dca_simt_kernel(
 // Candidate kernel (one block per candidate): YC = [X^C X^R^T, X^C X^C^T], OC = ZR + W_CC YC.
 // ---------------------------------------------------------------------------------------------
 template <typename T>
-__global__ void __launch_bounds__(128) glm_request_simt_kernel(
+__global__ void __launch_bounds__(256) glm_request_simt_kernel(
     int32_t n_r, int32_t n_c, int32_t d, const T* __restrict__ XR, const T* __restrict__ W,
     int32_t n_ro, int32_t n_co, T* __restrict__ YR, T* __restrict__ OR_, float* __restrict__ ZR) {
   extern __shared__ float sm[];
   const int32_t n = n_r + n_c;
-  float* xr = sm;                 // [n_r, d]
-  float* g = sm + (size_t)n_r * d;  // [n_r, n_r]
+  const int32_t ds = d + 1;                    // padded row stride: rows land in different banks
+  float* xr = sm;                              // [n_r, d + 1]
+  float* g = xr + (size_t)n_r * ds;            // [n_r, n_r]
+  float* w = g + (size_t)n_r * n_r;            // [n_ro + n_co, n_r]: the request columns of W
   const int32_t r = blockIdx.x;
-  for (int e = threadIdx.x; e < n_r * d; e += blockDim.x) xr[e] = ld_f(XR, (int64_t)r * n_r * d + e);
+  for (int e = threadIdx.x; e < n_r * d; e += blockDim.x)
+    xr[(e / d) * ds + e % d] = ld_f(XR, (int64_t)r * n_r * d + e);
+  if (W)
+    for (int e = threadIdx.x; e < (n_ro + n_co) * n_r; e += blockDim.x)
+      w[e] = ld_f(W, (int64_t)(e / n_r) * n + e % n_r);
   __syncthreads();
   for (int idx = threadIdx.x; idx < n_r * n_r; idx += blockDim.x) {
     const int a = idx / n_r, b = idx % n_r;
     float acc = 0.f;
-    for (int e = 0; e < d; ++e) acc = fmaf(xr[a * d + e], xr[b * d + e], acc);
+    for (int e = 0; e < d; ++e) acc = fmaf(xr[a * ds + e], xr[b * ds + e], acc);
     g[idx] = acc;
   }
   __syncthreads();
@@ -192,7 +198,7 @@ __global__ void __launch_bounds__(128) glm_request_simt_kernel(
       const int o = idx / n, b = idx % n;
       float acc = 0.f;
       if (b < n_r)
-        for (int a = 0; a < n_r; ++a) acc = fmaf(ld_f(W, (int64_t)o * n + a), g[a * n_r + b], acc);
+        for (int a = 0; a < n_r; ++a) acc = fmaf(w[o * n_r + a], g[a * n_r + b], acc);
       if (o < n_ro) {
         if (OR_) st_f(OR_, ((int64_t)r * n_ro + o) * n + b, acc);
       } else if (ZR) {
@@ -209,17 +215,19 @@ __global__ void __launch_bounds__(128) glm_candidate_simt_kernel(
     const float* __restrict__ ZR, T* __restrict__ YC, T* __restrict__ OC) {
   extern __shared__ float sm[];
   const int32_t n = n_r + n_c;
-  float* x = sm;                    // [n, d]: request rows then candidate rows
-  float* yc = sm + (size_t)n * d;   // [n_c, n]
+  const int32_t ds = d + 1;          // padded row stride: rows land in different banks
+  float* x = sm;                     // [n, d + 1]: request rows then candidate rows
+  float* yc = sm + (size_t)n * ds;   // [n_c, n]
   const int64_t i = blockIdx.x;
   const int32_t r = row2req[i];
-  for (int e = threadIdx.x; e < n_r * d; e += blockDim.x) x[e] = ld_f(XR, (int64_t)r * n_r * d + e);
-  for (int e = threadIdx.x; e < n_c * d; e += blockDim.x) x[n_r * d + e] = ld_f(XC, i * n_c * d + e);
+  for (int e = threadIdx.x; e < n_r * d; e += blockDim.x) x[(e / d) * ds + e % d] = ld_f(XR, (int64_t)r * n_r * d + e);
+  for (int e = threadIdx.x; e < n_c * d; e += blockDim.x)
+    x[(n_r + e / d) * ds + e % d] = ld_f(XC, i * n_c * d + e);
   __syncthreads();
   for (int idx = threadIdx.x; idx < n_c * n; idx += blockDim.x) {
     const int a = idx / n, b = idx % n;
-    const float* xa = x + (size_t)(n_r + a) * d;
-    const float* xb = x + (size_t)b * d;
+    const float* xa = x + (size_t)(n_r + a) * ds;
+    const float* xb = x + (size_t)b * ds;
     float acc = 0.f;
     for (int e = 0; e < d; ++e) acc = fmaf(xa[e], xb[e], acc);
     yc[idx] = acc;
@@ -279,14 +287,14 @@ static rocs_status_t launch_glm(const rocs_plan* plan, int32_t n_r, int32_t n_c,
                                 int32_t n_co, void* YR, void* YC, void* OR_, void* OC, float* zr,
                                 bool request_side, bool candidate_side, cudaStream_t stream) {
   const int32_t n = n_r + n_c;
-  const size_t smem_r = ((size_t)n_r * d + (size_t)n_r * n_r) * sizeof(float);
-  const size_t smem_c = ((size_t)n * d + (size_t)n_c * n) * sizeof(float);
+  const size_t smem_r = ((size_t)n_r * (d + 1) + (size_t)n_r * n_r + (size_t)(n_ro + n_co) * n_r) * sizeof(float);
+  const size_t smem_c = ((size_t)n * (d + 1) + (size_t)n_c * n) * sizeof(float);
   constexpr size_t kMaxSmem = 200 * 1024;
   if (smem_r > kMaxSmem || smem_c > kMaxSmem) return ROCS_ERR_UNSUPPORTED;
   if (request_side && plan->R > 0) {
     ROCS_CUDA_TRY(cudaFuncSetAttribute(glm_request_simt_kernel<T>,
                                        cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kMaxSmem));
-    glm_request_simt_kernel<T><<<plan->R, 128, smem_r, stream>>>(
+    glm_request_simt_kernel<T><<<plan->R, 256, smem_r, stream>>>(
         n_r, n_c, d, (const T*)XR, (const T*)W, n_ro, n_co, (T*)YR, (T*)OR_, zr);
     ROCS_CUDA_TRY(cudaGetLastError());
   }
