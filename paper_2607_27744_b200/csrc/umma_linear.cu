@@ -312,6 +312,8 @@ rocs_status_t umma_linear(int64_t M, int32_t d_in, int32_t d_out, const void* X,
                           int64_t ld_w, const float* bias, const float* add, int64_t ld_add,
                           const int32_t* row2req, int act, void* Y, int64_t ld_y, bool out_f32,
                           cudaStream_t stream) {
+  if (umma_linear_ws2_supported(M, d_in, d_out, out_f32))
+    return umma_linear_ws2(M, d_in, d_out, X, ld_x, W, ld_w, bias, add, ld_add, row2req, act, Y, ld_y, stream);
   if (umma_linear_ws_supported(M, d_in, d_out, out_f32))
     return umma_linear_ws(M, d_in, d_out, X, ld_x, W, ld_w, bias, add, ld_add, row2req, act, Y, ld_y, stream);
 #define ROCS_LAUNCH(BN_)                                                                                   \

@@ -31,6 +31,7 @@ constexpr int kEpiWarps = 8;
 constexpr int kAStageBytes = BM * BK * 2;   // 16 KB
 constexpr int kWBlockBytes = BN * BK * 2;   // 32 KB per 64-wide K block
 constexpr int kZBufBytes = 4 * BN * 4;      // four slabs x 256 fp32
+constexpr int kZBufs = 4;                   // request-row buffers: the producer may run this many tiles ahead
 constexpr uint32_t kStatusWs = 0x300;
 
 struct WsParams {
@@ -55,14 +56,14 @@ linear_ws_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constan
   const int32_t k_blocks = (p.d_in + BK - 1) / BK;
   uint8_t* w_smem = smem;
   uint8_t* a_smem = w_smem + k_blocks * kWBlockBytes;
-  float* z_smem = reinterpret_cast<float*>(a_smem + p.a_stages * kAStageBytes);  // [2][4][256]
-  uint64_t* a_full = reinterpret_cast<uint64_t*>(reinterpret_cast<uint8_t*>(z_smem) + 2 * kZBufBytes);
+  float* z_smem = reinterpret_cast<float*>(a_smem + p.a_stages * kAStageBytes);  // [kZBufs][4][256]
+  uint64_t* a_full = reinterpret_cast<uint64_t*>(reinterpret_cast<uint8_t*>(z_smem) + kZBufs * kZBufBytes);
   uint64_t* a_empty = a_full + 8;
   uint64_t* tmem_full = a_empty + 8;
   uint64_t* tmem_empty = tmem_full + 2;
   uint64_t* z_full = tmem_empty + 2;
-  uint64_t* z_empty = z_full + 2;
-  uint64_t* w_full = z_empty + 2;
+  uint64_t* z_empty = z_full + kZBufs;
+  uint64_t* w_full = z_empty + kZBufs;
   uint64_t* drain = w_full + 1;
   uint32_t* tmem_ptr = reinterpret_cast<uint32_t*>(drain + 1);
   AbortFlag* abort_flag = reinterpret_cast<AbortFlag*>(tmem_ptr + 1);
@@ -81,6 +82,8 @@ linear_ws_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constan
     for (int a = 0; a < 2; ++a) {
       mbar_init(&tmem_full[a], 1);
       mbar_init(&tmem_empty[a], kEpiWarps);
+    }
+    for (int a = 0; a < kZBufs; ++a) {
       mbar_init(&z_full[a], 1);
       mbar_init(&z_empty[a], kEpiWarps);
     }
@@ -107,26 +110,33 @@ linear_ws_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constan
       for (int32_t kb = 0; kb < k_blocks; ++kb) tma_load_2d(w_smem + kb * kWBlockBytes, &map_w, w_full, kb * BK, n0);
       uint32_t it = 0, lt = 0;
       bool ok = true;
+      // request ids of the four slabs of a tile, fetched one tile ahead of their use
+      int32_t req_next[4] = {0, 0, 0, 0};
+      auto fetch_req = [&](int32_t mt_) {
+#pragma unroll
+        for (int q = 0; q < 4; ++q) {
+          const int64_t r0 = min((int64_t)mt_ * BM + q * 32, p.M - 1);
+          req_next[q] = p.row2req ? p.row2req[r0] : (int32_t)r0;
+        }
+      };
+      if (has_add && group < m_tiles) fetch_req(group);
       for (int32_t mt = group; mt < m_tiles && ok; mt += p.groups, ++lt) {
         const int32_t m0 = mt * BM;
-        if (has_add) {
-          const uint32_t zb = lt & 1;
-          if (!mbar_wait(&z_empty[zb], ((lt >> 1) & 1) ^ 1, abort_flag, p.status, kStatusWs | 5)) { ok = false; break; }
-          mbar_expect_tx(&z_full[zb], kZBufBytes);
-          int32_t req[4];
-#pragma unroll
-          for (int q = 0; q < 4; ++q) {
-            const int64_t r0 = min((int64_t)m0 + q * 32, p.M - 1);
-            req[q] = p.row2req ? p.row2req[r0] : (int32_t)r0;
-          }
-#pragma unroll
-          for (int q = 0; q < 4; ++q) tma_load_2d(z_smem + (zb * 4 + q) * BN, &map_z, &z_full[zb], n0, req[q]);
-        }
+        // X first: the MMA needs it now; the request rows are only needed by this tile's epilogue
         for (int32_t kb = 0; kb < k_blocks; ++kb, ++it) {
           const int s = it % p.a_stages;
           if (!mbar_wait(&a_empty[s], ((it / p.a_stages) & 1) ^ 1, abort_flag, p.status, kStatusWs | 1)) { ok = false; break; }
           mbar_expect_tx(&a_full[s], kAStageBytes);
           tma_load_2d(a_smem + s * kAStageBytes, &map_x, &a_full[s], kb * BK, m0);
+        }
+        if (!ok) break;
+        if (has_add) {
+          const uint32_t zb = lt % kZBufs;
+          if (!mbar_wait(&z_empty[zb], ((lt / kZBufs) & 1) ^ 1, abort_flag, p.status, kStatusWs | 5)) { ok = false; break; }
+          mbar_expect_tx(&z_full[zb], kZBufBytes);
+#pragma unroll
+          for (int q = 0; q < 4; ++q) tma_load_2d(z_smem + (zb * 4 + q) * BN, &map_z, &z_full[zb], n0, req_next[q]);
+          if (mt + p.groups < m_tiles) fetch_req(mt + p.groups);
         }
       }
       if (!ok) {
@@ -186,8 +196,8 @@ linear_ws_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constan
         const int32_t my_req = p.row2req ? p.row2req[rc] : (int32_t)rc;
         const int32_t slab_req = __shfl_sync(0xffffffffu, my_req, 0);
         // shared-memory copy when this row belongs to the slab's first request, global otherwise
-        zrow = (my_req == slab_req) ? (z_smem + (acc * 4 + q) * BN) : (p.add + (int64_t)my_req * p.ld_add + n0);
-        if (!mbar_wait(&z_full[acc], (lt >> 1) & 1, abort_flag, p.status, kStatusWs | 7)) break;
+        zrow = (my_req == slab_req) ? (z_smem + ((lt % kZBufs) * 4 + q) * BN) : (p.add + (int64_t)my_req * p.ld_add + n0);
+        if (!mbar_wait(&z_full[lt % kZBufs], (lt / kZBufs) & 1, abort_flag, p.status, kStatusWs | 7)) break;
       }
       if (!mbar_wait(&tmem_full[acc], (lt >> 1) & 1, abort_flag, p.status, kStatusWs | 4)) break;
       tc_fence_after_sync();
@@ -256,7 +266,7 @@ linear_ws_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constan
       }
       if (has_add) {
         __syncwarp();
-        if (lane == 0) mbar_arrive(&z_empty[acc]);
+        if (lane == 0) mbar_arrive(&z_empty[lt % kZBufs]);
       }
     }
   }
@@ -313,7 +323,7 @@ rocs_status_t umma_linear_ws(int64_t M, int32_t d_in, int32_t d_out, const void*
   p.n_slices = (d_out + BN - 1) / BN;
   const int32_t m_tiles = (int32_t)((M + BM - 1) / BM);
   p.groups = std::max(1, std::min(m_tiles, sm_count_ws() / p.n_slices));
-  const int fixed = k_blocks * kWBlockBytes + 2 * kZBufBytes + 512 + 1024;
+  const int fixed = k_blocks * kWBlockBytes + kZBufs * kZBufBytes + 512 + 1024;
   p.a_stages = std::min(8, (227 * 1024 - fixed) / kAStageBytes);
   p.bias = bias; p.add = add; p.ld_add = ld_add; p.row2req = row2req; p.act = act;
   p.Y = (__nv_bfloat16*)Y; p.ld_y = ld_y; p.status = status;
