@@ -18,7 +18,6 @@
 //                       registers, + Z (shared-memory broadcast when the slab has one request,
 //                       global gather otherwise), ReLU, bf16, swizzled staging, TMA store
 #include <algorithm>
-#include <cstdlib>
 
 #include "rocs_internal.h"
 #include "sm100_ptx.cuh"
@@ -48,7 +47,6 @@ struct Ws2Params {
   const int32_t* row2req;
   int32_t act;
   uint32_t* status;
-  int32_t dbg;
 };
 
 __device__ __forceinline__ float4 lds128(const float* p) {
@@ -238,7 +236,7 @@ linear_ws2_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_consta
         float f[64];
 #pragma unroll
         for (int i = 0; i < 64; ++i) f[i] = __uint_as_float(v[i]);
-        if (has_add && !(p.dbg & 1)) {
+        if (has_add) {
           if (uniform) {
 #pragma unroll
             for (int i = 0; i < 64; i += 4) {  // one broadcast read per 16 bytes (columns past d_out hold zeros)
@@ -283,13 +281,13 @@ linear_ws2_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_consta
           *reinterpret_cast<uint4*>(row_ptr + ((j ^ (lane & 7)) << 4)) = w;
         }
       }
-      if (!(p.dbg & 8)) fence_proxy_async_smem();
+      fence_proxy_async_smem();
       __syncwarp();
       if (lane == 0) {
 #pragma unroll
         for (int c = 0; c < 2; ++c)
-          if (n0 + half * 128 + c * 64 < p.d_out && (int64_t)m0 + q * 32 < p.M && !(p.dbg & 2))
-            tma_store_2d(&map_y, my_stage + c * 4096, n0 + half * 128 + c * 64, (p.dbg & 4) ? (int32_t)(rank * BM + q * 32) : m0 + q * 32);
+          if (n0 + half * 128 + c * 64 < p.d_out && (int64_t)m0 + q * 32 < p.M)
+            tma_store_2d(&map_y, my_stage + c * 4096, n0 + half * 128 + c * 64, m0 + q * 32);
         tma_store_commit();
         if (has_add) mbar_arrive(&z_empty[lt % kZBufs]);
       }
@@ -351,8 +349,6 @@ rocs_status_t umma_linear_ws2(int64_t M, int32_t d_in, int32_t d_out, const void
   p.groups = std::max(1, std::min(super_tiles, (sm_count_ws2() / 2) / p.n_slices));
   const int fixed = k_blocks * kWBlockBytes + kStagingBytes + kZBufs * kZBufBytes + 512 + 1024;
   p.a_stages = std::min(10, (227 * 1024 - fixed) / kAStageBytes);
-  { static const char* e2 = getenv("ROCS_LINEAR_DEBUG"); p.dbg = e2 ? atoi(e2) : 0; }
-  { static const char* e = getenv("ROCS_WS2_STAGES"); if (e) p.a_stages = std::min(p.a_stages, atoi(e)); }
   p.bias = bias; p.add = add; p.ld_add = ld_add; p.row2req = row2req; p.act = act; p.status = status;
   const int smem_bytes = fixed + p.a_stages * kAStageBytes;
   ROCS_CUDA_TRY(cudaFuncSetAttribute(linear_ws2_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_bytes));
