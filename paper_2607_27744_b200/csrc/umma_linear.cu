@@ -321,8 +321,14 @@ rocs_status_t umma_linear(int64_t M, int32_t d_in, int32_t d_out, const void* X,
                                 stream)                                                                    \
            : launch<BN_, __nv_bfloat16>(M, d_in, d_out, X, ld_x, W, ld_w, bias, add, ld_add, row2req, act, Y, \
                                         ld_y, stream))
-  if (d_out > 128) return ROCS_LAUNCH(256);
-  if (d_out > 64) return ROCS_LAUNCH(128);
+  // Widest tile that still gives every SM something to do: a small batch (the request half at
+  // batch size R) is spread over more, narrower tiles instead of leaving most SMs idle.
+  const int64_t m_tiles = (M + BM - 1) / BM;
+  const int sms = sm_count();
+  int bn = d_out > 128 ? 256 : (d_out > 64 ? 128 : 64);
+  while (bn > 64 && m_tiles * ((d_out + bn - 1) / bn) < sms) bn /= 2;
+  if (bn == 256) return ROCS_LAUNCH(256);
+  if (bn == 128) return ROCS_LAUNCH(128);
   return ROCS_LAUNCH(64);
 #undef ROCS_LAUNCH
 }
