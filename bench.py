@@ -35,6 +35,10 @@ METRIC = "candidates scored/sec per IKBO layer (bf16, 1 B200) and % of roofline"
 UNIT = "candidates/s"
 WORKLOAD = "config 2: retrieval MLP bf16, R=256 x 512 candidates (N=131072), 768->1024->1024->256, layer 1 split 512|256"
 N_SETS = 4  # rotating input/output sets: 4 x (67 MB in + 600 MB activations) >> 126 MB L2
+# dram__bytes_read.sum + dram__bytes_write.sum per launch, from the ncu captures summarised under
+# profiles/ (bytes; the request half of layer 1 adds 1.3 MB).  Below the algorithmic bytes where the
+# tail of the output is still in L2 when the kernel ends.
+NCU_TRAFFIC = {"L1": 283.9e6 + 1.3e6, "L2": 495.6e6, "L3": 315.6e6}
 
 
 def measured_peaks():
@@ -205,13 +209,23 @@ def run_rocs(args):
     workspace = torch.empty(ws_bytes, dtype=torch.uint8, device="cuda")
     launches_per_step = 5  # fill_row2req, request half, candidate half, layer 2, layer 3
 
-    def step(i, XR=None, XC=None, co_d=None):
+    def step(i, XR=None, XC=None, co_d=None, marks=None):
         s = i % N_SETS
+        if marks is not None:
+            marks[0].record()
         plan = rocs.plan_create(co_dev if co_d is None else co_d, co)
+        if marks is not None:
+            marks[1].record()
         rocs.ikbo_linear(plan, XR_sets[s] if XR is None else XR, XC_sets[s] if XC is None else XC, W1_cr, W1_cc,
                          relu=True, out=h1[s], workspace=workspace)
+        if marks is not None:
+            marks[2].record()
         rocs.linear(h1[s], W2, relu=True, out=h2[s])
+        if marks is not None:
+            marks[3].record()
         rocs.linear(h2[s], W3, out=y[s])
+        if marks is not None:
+            marks[4].record()
         plan.close()
         return y[s]
 
@@ -236,10 +250,13 @@ def run_rocs(args):
         step(i)
     barrier()
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    # events between the calls of every timed step: per-layer durations measured INSIDE the timed
+    # region, on the stream the kernels run on (they cost a few hundred ns each)
+    marks = [[torch.cuda.Event(enable_timing=True) for _ in range(5)] for _ in range(args.steps)]
     with ClockSampler(local) as clocks:
         e0.record()
         for i in range(args.steps):
-            step(i)
+            step(i, marks=marks[i])
         e1.record()
         barrier()
         if ms_estimate(e0, e1) < 600.0:   # keep the same load running until a few clock samples exist
@@ -254,7 +271,12 @@ def run_rocs(args):
     ms_per_step = ms / args.steps
     value = world * N / (ms_per_step * 1e-3)
 
-    # ---- per-layer timing (CUDA events around each call, same rotating sets) -----------------
+    # ---- per-layer durations inside the timed region ------------------------------------------
+    def span(a, b):
+        return float(np.mean([m[a].elapsed_time(m[b]) for m in marks])) * 1e-3
+
+    t_plan_in, t_l1, t_l2, t_l3 = span(0, 1), span(1, 2), span(2, 3), span(3, 4)
+
     def time_call(fn, reps=20):
         for i in range(3):
             fn(i)
@@ -267,35 +289,39 @@ def run_rocs(args):
         torch.cuda.synchronize()
         return a.elapsed_time(b) / reps * 1e-3
 
-    plan = rocs.plan_create(co_dev, co)
-    t_l1 = time_call(lambda i: rocs.ikbo_linear(plan, XR_sets[i % N_SETS], XC_sets[i % N_SETS], W1_cr, W1_cc, relu=True,
-                                                out=h1[i % N_SETS], workspace=workspace))
-    t_l2 = time_call(lambda i: rocs.linear(h1[i % N_SETS], W2, relu=True, out=h2[i % N_SETS]))
-    t_l3 = time_call(lambda i: rocs.linear(h2[i % N_SETS], W3, out=y[i % N_SETS]))
     t_plan = time_call(lambda i: rocs.plan_create(co_dev, co).close())
 
-    def layer(name, t, flops, nbytes):
+    def layer(name, t, flops, nbytes, traffic):
+        # These durations come from inside the long timed step, so a tensor-bound layer is held
+        # against the SUSTAINED measured bf16 peak (the burst figure is given beside it).
         t_hbm = nbytes / (peaks["hbm_gbs"] * 1e9)
-        t_tc = flops / (peaks["tflops_burst"] * 1e12)
+        t_tc = flops / (peaks["tflops_sustained"] * 1e12)
         bound = "hbm" if t_hbm >= t_tc else "tensor"
         ach = nbytes / t / 1e9 if bound == "hbm" else flops / t / 1e12
-        peak = peaks["hbm_gbs"] if bound == "hbm" else peaks["tflops_burst"]
+        peak = peaks["hbm_gbs"] if bound == "hbm" else peaks["tflops_sustained"]
         return {"layer": name, "us": t * 1e6, "cand_per_s": N / t, "bound": bound, "achieved": ach, "peak": peak,
                 "unit": "GB/s" if bound == "hbm" else "TFLOP/s", "frac": ach / peak,
-                "tflops": flops / t / 1e12, "gbs": nbytes / t / 1e9}
+                "tflops": flops / t / 1e12, "gbs": nbytes / t / 1e9,
+                "frac_of_burst_tensor_peak": flops / t / 1e12 / peaks["tflops_burst"],
+                "algorithmic_bytes": nbytes, "traffic": traffic}
 
     bf = 2
     layers = [
         layer("cfg2.L1 ikbo_linear 512|256->1024 (request half + candidate half)", t_l1,
               2.0 * N * 256 * 1024 + 2.0 * 256 * 512 * 1024,
-              N * 256 * bf + N * 1024 * bf + 256 * 512 * bf + 1024 * 768 * bf),
-        layer("cfg2.L2 linear 1024->1024", t_l2, 2.0 * N * 1024 * 1024, N * 1024 * bf * 2 + 1024 * 1024 * bf),
-        layer("cfg2.L3 linear 1024->256", t_l3, 2.0 * N * 1024 * 256, N * 1024 * bf + N * 256 * bf + 256 * 1024 * bf),
+              N * 256 * bf + N * 1024 * bf + 256 * 512 * bf + 1024 * 768 * bf, NCU_TRAFFIC["L1"]),
+        layer("cfg2.L2 linear 1024->1024", t_l2, 2.0 * N * 1024 * 1024, N * 1024 * bf * 2 + 1024 * 1024 * bf,
+              NCU_TRAFFIC["L2"]),
+        layer("cfg2.L3 linear 1024->256", t_l3, 2.0 * N * 1024 * 256, N * 1024 * bf + N * 256 * bf + 256 * 1024 * bf,
+              NCU_TRAFFIC["L3"]),
     ]
     dominant = max(layers, key=lambda l: l["us"])
     roofline = {"kernel": dominant["layer"], "bound": dominant["bound"], "achieved": dominant["achieved"],
-                "peak": dominant["peak"], "unit": dominant["unit"], "frac": dominant["frac"], "traffic": None,
-                "peak_source": peaks["source"] + (" (burst)" if dominant["bound"] == "tensor" else "")}
+                "peak": dominant["peak"], "unit": dominant["unit"], "frac": dominant["frac"],
+                "traffic": dominant["traffic"],
+                "peak_source": "of " + peaks["source"] + (" (sustained; timed inside the step)"
+                                                          if dominant["bound"] == "tensor" else ""),
+                "timed": "CUDA events between the calls of every timed step"}
 
     # ---- attention and interaction kernels on their own workloads ----------------------------
     extra = []
@@ -346,7 +372,7 @@ def run_rocs(args):
         "roofline": roofline,
         "cpu_baseline": cpu,
         "layers": layers,
-        "plan_us": t_plan * 1e6,
+        "plan_us": t_plan * 1e6, "plan_us_in_step": t_plan_in * 1e6,
         "other_ikbo_layers": extra,
     }))
 
@@ -376,7 +402,10 @@ def bench_dca(torch, rocs, peaks, dev, time_call):
     nbytes = (2 * Q.numel() + 2 * K.numel()) * 2
     return {"layer": "cfg3 dca_attention (R=64, L=2048, 8x64)", "N": N, "us": t * 1e6, "cand_per_s": N / t,
             "tflops": flops / t / 1e12, "frac_tensor": flops / t / 1e12 / peaks["tflops_burst"],
-            "gbs": nbytes / t / 1e9, "exps_per_s": pairs * cfg.H / t}
+            "gbs": nbytes / t / 1e9, "exps_per_s": pairs * cfg.H / t,
+            "bound": "tensor (nominal); the exponential unit (16 ex2/clk/SM) is the tighter ceiling at dh = 64",
+            "frac_of_exp_unit_peak_at_max_clock": pairs * cfg.H / t / (148 * 16 * 1.965e9),
+            "frac_tensor_sustained": flops / t / 1e12 / peaks["tflops_sustained"]}
 
 
 def bench_glm(torch, rocs, peaks, dev, time_call):
