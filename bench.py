@@ -323,6 +323,12 @@ def run_rocs(args):
                                                           if dominant["bound"] == "tensor" else ""),
                 "timed": "CUDA events between the calls of every timed step"}
 
+    # ---- materialised-broadcast GPU path for the IKBO layer (reference point) ------------------
+    counts_dev = dev(np.diff(co).astype(np.int64))
+    t_mat = time_call(lambda i: materialised_linear(torch, XR_sets[i % N_SETS], XC_sets[i % N_SETS], W1, counts_dev), reps=10)
+    layers[0]["materialised_broadcast_gpu_us"] = t_mat * 1e6
+    layers[0]["speedup_vs_materialised"] = t_mat / t_l1
+
     # ---- attention and interaction kernels on their own workloads ----------------------------
     extra = []
     if not args.skip_extra:
@@ -384,7 +390,49 @@ def bench_other_ops(torch, rocs, peaks, dev, time_call, which=("dca", "glm")):
         out.append(bench_dca(torch, rocs, peaks, dev, time_call))
     if "glm" in which:
         out.append(bench_glm(torch, rocs, peaks, dev, time_call))
+    if "cfg5" in which:
+        out.extend(bench_cfg5(torch, rocs, peaks, dev, time_call))
     return out
+
+
+def materialised_linear(torch, XR, XC, W, counts_dev, relu=True):
+    """The dense path the paper starts from (Section 4, first paragraph): replicate the request rows
+    per candidate, concatenate, one full GEMM.  torch library kernels; a reference point only."""
+    u = torch.cat([XR.repeat_interleave(counts_dev, dim=0), XC], dim=1)
+    y = u @ W.t()
+    return torch.relu_(y) if relu else y
+
+
+def materialised_dca(torch, Q, K, V, co, so, chunk_bytes=4 << 30):
+    """Candidate-batched copies of K/V, then library attention (Section 4.3, second paragraph),
+    request by request in chunks so the copies fit in memory."""
+    N, n_q, H, dh = Q.shape
+    O = torch.empty_like(Q)
+    for r in range(len(co) - 1):
+        c0, c1, s0, s1 = int(co[r]), int(co[r + 1]), int(so[r]), int(so[r + 1])
+        if c1 == c0 or s1 == s0:
+            continue
+        per_cand = 2 * (s1 - s0) * H * dh * 2
+        step = max(1, int(chunk_bytes // per_cand))
+        k = K[s0:s1].permute(1, 0, 2)  # [H, L, dh]
+        v = V[s0:s1].permute(1, 0, 2)
+        for a in range(c0, c1, step):
+            b = min(c1, a + step)
+            kk = k.unsqueeze(0).expand(b - a, -1, -1, -1).contiguous()   # the materialised broadcast
+            vv = v.unsqueeze(0).expand(b - a, -1, -1, -1).contiguous()
+            q = Q[a:b].permute(0, 2, 1, 3)
+            O[a:b] = torch.nn.functional.scaled_dot_product_attention(q, kk, vv).permute(0, 2, 1, 3)
+    return O
+
+
+def materialised_glm(torch, XR, XC, W, counts_dev, n_r, n_ro):
+    """X = [X^R[m_i]; X^C[i]] per candidate, G = X X^T, block mask, O = W~ G (Eq. 9-10, Eq. 5-6)."""
+    X = torch.cat([XR.repeat_interleave(counts_dev, dim=0), XC], dim=1)
+    G = torch.bmm(X, X.transpose(1, 2))
+    G[:, :n_r, n_r:] = 0
+    Wm = W.clone()
+    Wm[:n_ro, n_r:] = 0
+    return torch.matmul(Wm, G)
 
 
 def bench_dca(torch, rocs, peaks, dev, time_call):
@@ -400,7 +448,9 @@ def bench_dca(torch, rocs, peaks, dev, time_call):
     pairs = float(np.sum(np.diff(co).astype(np.float64) * np.diff(so)))
     flops = 4.0 * pairs * cfg.H * cfg.dh
     nbytes = (2 * Q.numel() + 2 * K.numel()) * 2
+    t_mat = time_call(lambda i: materialised_dca(torch, Q, K, V, co, so), reps=1)
     return {"layer": "cfg3 dca_attention (R=64, L=2048, 8x64)", "N": N, "us": t * 1e6, "cand_per_s": N / t,
+            "materialised_broadcast_gpu_us": t_mat * 1e6, "speedup_vs_materialised": t_mat / t,
             "tflops": flops / t / 1e12, "frac_tensor": flops / t / 1e12 / peaks["tflops_burst"],
             "gbs": nbytes / t / 1e9, "exps_per_s": pairs * cfg.H / t,
             "bound": "tensor (nominal); the exponential unit (16 ex2/clk/SM) is the tighter ceiling at dh = 64",
@@ -424,10 +474,59 @@ def bench_glm(torch, rocs, peaks, dev, time_call):
                                                  outs=outs), reps=10)
     nbytes = XC.numel() * 2 + outs["OC"].numel() * 2 + XR.numel() * 2
     flops = N * (2.0 * cfg.n_c * n * cfg.d_emb + 2.0 * cfg.n_co * cfg.n_c * n)
+    counts_dev = dev(np.diff(co).astype(np.int64))
+    t_mat = time_call(lambda i: materialised_glm(torch, XR, XC, W, counts_dev, cfg.n_r, cfg.n_ro), reps=3)
     return {"layer": "cfg4 glm_interaction 32+16 x128, 48->16 compression (OC only)", "N": N, "us": t * 1e6,
+            "materialised_broadcast_gpu_us": t_mat * 1e6, "speedup_vs_materialised": t_mat / t,
             "cand_per_s": N / t, "gbs": nbytes / t / 1e9, "frac_hbm": nbytes / t / 1e9 / peaks["hbm_gbs"],
             "tflops": flops / t / 1e12,
             "note": "input (537 MB) is larger than L2; same buffers every iteration"}
+
+
+def bench_cfg5(torch, rocs, peaks, dev, time_call):
+    """Configuration 5 (skewed, Zipf candidate counts): the three calls timed independently."""
+    cfg = wl.CONFIGS[5]
+    co, so = wl.cand_offsets(cfg), wl.seq_offsets(cfg)
+    N = int(co[-1])
+    plan = rocs.plan_create(dev(co), co)
+    out = []
+    g = torch.Generator(device="cuda").manual_seed(5)
+    rnd = lambda *shape: torch.randn(*shape, generator=g, device="cuda", dtype=torch.float32).to(torch.bfloat16)
+    # linear 768|256 -> 1024
+    XR, XC = rnd(cfg.R, cfg.d_req), rnd(N, cfg.d_cand)
+    W = (rnd(cfg.d_out, cfg.d_req + cfg.d_cand).float() / 32).to(torch.bfloat16)
+    Y = torch.empty((N, cfg.d_out), dtype=torch.bfloat16, device="cuda")
+    ws = torch.empty(rocs.ikbo_linear_workspace(plan, cfg.d_out), dtype=torch.uint8, device="cuda")
+    t = time_call(lambda i: rocs.ikbo_linear(plan, XR, XC, W[:, :cfg.d_req], W[:, cfg.d_req:], out=Y, workspace=ws), reps=5)
+    nbytes = (XC.numel() + Y.numel() + XR.numel() + W.numel()) * 2
+    counts_dev = dev(np.diff(co).astype(np.int64))
+    t_mat = time_call(lambda i: materialised_linear(torch, XR, XC, W, counts_dev, relu=False), reps=2)
+    out.append({"layer": "cfg5 ikbo_linear 768|256->1024 (Zipf segments)", "N": N, "us": t * 1e6, "cand_per_s": N / t,
+                "gbs": nbytes / t / 1e9, "frac_hbm": nbytes / t / 1e9 / peaks["hbm_gbs"],
+                "materialised_broadcast_gpu_us": t_mat * 1e6, "speedup_vs_materialised": t_mat / t})
+    del XC, Y
+    # attention, L in [256, 1024]
+    T = int(so[-1])
+    Q, K, V = rnd(N, 1, cfg.H, cfg.dh), rnd(T, cfg.H, cfg.dh), rnd(T, cfg.H, cfg.dh)
+    O = torch.empty_like(Q)
+    sod = dev(so)
+    t = time_call(lambda i: rocs.dca_attention(plan, Q, K, V, sod, out=O), reps=3)
+    pairs = float(np.sum(np.diff(co).astype(np.float64) * np.diff(so)))
+    flops = 4.0 * pairs * cfg.H * cfg.dh
+    out.append({"layer": "cfg5 dca_attention (Zipf segments, L in [256,1024], 8x64)", "N": N, "us": t * 1e6,
+                "cand_per_s": N / t, "tflops": flops / t / 1e12, "frac_tensor": flops / t / 1e12 / peaks["tflops_burst"],
+                "exps_per_s": pairs * cfg.H / t})
+    del Q, K, V, O
+    # interaction 24 + 8, no compression
+    GR, GC = rnd(cfg.R, cfg.n_r, cfg.d_emb), rnd(N, cfg.n_c, cfg.d_emb)
+    n = cfg.n_r + cfg.n_c
+    outs = {"YC": torch.empty((N, cfg.n_c, n), dtype=torch.bfloat16, device="cuda"),
+            "YR": torch.empty((cfg.R, cfg.n_r, n), dtype=torch.bfloat16, device="cuda")}
+    t = time_call(lambda i: rocs.glm_interaction(plan, GR, GC, None, 0, 0, want_raw=True, outs=outs), reps=5)
+    nbytes = (GC.numel() + outs["YC"].numel()) * 2
+    out.append({"layer": "cfg5 glm_interaction 24+8 x128 (raw YC)", "N": N, "us": t * 1e6, "cand_per_s": N / t,
+                "gbs": nbytes / t / 1e9, "frac_hbm": nbytes / t / 1e9 / peaks["hbm_gbs"]})
+    return out
 
 
 def main():
@@ -437,7 +536,7 @@ def main():
     ap.add_argument("--warmup", type=int, default=10)
     ap.add_argument("--impl", default="rocs", choices=["rocs", "reference"])
     ap.add_argument("--skip-extra", action="store_true", help="skip the attention / interaction side measurements")
-    ap.add_argument("--extra", default="dca,glm", help="which side measurements to run (dca, glm)")
+    ap.add_argument("--extra", default="dca,glm", help="side measurements to run: dca, glm, cfg5")
     ap.add_argument("--skip-cpu", action="store_true", help="skip the cpu_baseline leg")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "rocs" else args.warmup
