@@ -2,13 +2,14 @@
 // kernel (Section 4.3.1):  O[i,t,h,:] = softmax_j(scale <Q[i,t,h,:], K[r,j,h,:]>) V[r,j,h,:],  r = m_i.
 //
 // Candidates of one request are stacked in the tile M dimension: a work item is one head of up to
-// TWO 128-row query tiles (A and B) of the same request, so every 128-key block of K and V is loaded
+// TWO 128-row query tiles (A and B) of the same request, so every 64-key block of K and V is loaded
 // once and used by 256 query rows.  K/V are addressed per request through seq_offsets; nothing is
 // replicated per candidate.
 //
-// One persistent CTA per SM, 10 warps:
-//   warp 0     TMA producer: Q tiles of the item, then (K_j, V_j) blocks through a ring
-//   warp 1     tcgen05.mma issuer:  S_X = Q_X K_j^T  (128x128x64)  and  O_X = P_X V_j  (128x64x128)
+// Two persistent CTAs per SM (half the shared memory and half the TMEM columns each), so sixteen
+// softmax warps keep the exponential unit fed while others wait on barriers.  Per CTA, 10 warps:
+//   warp 0     TMA producer: Q tiles of the item, then (K_j, V_j) blocks of 64 keys through a ring
+//   warp 1     tcgen05.mma issuer:  S_X = Q_X K_j^T  (128x64x64)  and  O_X = P_X V_j  (128x64x64)
 //   warps 2-5  softmax group A,  warps 6-9  softmax group B: each thread owns one query row:
 //              S from TMEM into registers (one read), reference max and sum in fp32 (exp2 on scaled
 //              scores), P rounded to bf16 into shared memory (the A operand of the second MMA),
@@ -32,17 +33,19 @@ using namespace ptx;
 
 constexpr int DH = 64;            // head dimension handled here (128-byte rows)
 constexpr int BQ = 128;           // query rows per tile
-constexpr int BKV = 128;          // keys per block
+constexpr int BKV = 64;           // keys per block
 constexpr int kThreads = 320;
 constexpr int kKvStages = 3;
+constexpr int kQSlots = 1;        // Q buffers per side (the second CTA on the SM covers the item change-over)
+constexpr int kTmemCols = 256;    // per CTA; two CTAs share an SM
 constexpr int kQBytes = BQ * DH * 2;          // 16 KB
-constexpr int kKvStageBytes = 2 * BKV * DH * 2;  // K block + V block = 32 KB
-constexpr int kPBytes = BQ * BKV * 2;         // 32 KB per side
-constexpr int kSmemBytes = 4 * kQBytes + kKvStages * kKvStageBytes + 2 * kPBytes + 512 + 1024;
+constexpr int kKvStageBytes = 2 * BKV * DH * 2;  // K block + V block = 16 KB
+constexpr int kPBytes = BQ * BKV * 2;         // 16 KB per side
+constexpr int kSmemBytes = 2 * kQSlots * kQBytes + kKvStages * kKvStageBytes + 2 * kPBytes + 512;  // 1024-aligned base
 constexpr float kRescaleThreshold = 8.f;  // log2 units
 constexpr uint32_t kStatusDca = 0x400;
-constexpr int kSideTmemStride = 256;  // side A: columns 0.., side B: columns 256..
-constexpr int kOColOffset = 128;      // S in [0, 128), O block in [128, 192) of the side
+constexpr int kSideTmemStride = 128;  // side A: columns 0.., side B: columns 128..
+constexpr int kOColOffset = BKV;      // S in [0, 64), O block in [64, 128) of the side
 
 struct DcaParams {
   const DcaItem* items;
@@ -61,14 +64,13 @@ __device__ __forceinline__ float ex2(float x) {
   return y;
 }
 
-__global__ void __launch_bounds__(kThreads, 1)
+__global__ void __launch_bounds__(kThreads, 2)
 dca_umma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
                 const __grid_constant__ CUtensorMap map_v, const DcaParams p) {
-  extern __shared__ uint8_t smem_raw[];
-  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
-  uint8_t* q_smem = smem;                              // [2 slots][2 sides][128][64] bf16
-  uint8_t* kv_smem = q_smem + 4 * kQBytes;             // [stages][K 16 KB | V 16 KB]
-  uint8_t* p_smem = kv_smem + kKvStages * kKvStageBytes;  // [2][2 x (128 x 64)] bf16, K-major swizzled
+  extern __shared__ __align__(1024) uint8_t smem[];     // swizzled operand tiles need 1024-byte alignment
+  uint8_t* q_smem = smem;                              // [slots][2 sides][128][64] bf16
+  uint8_t* kv_smem = q_smem + 2 * kQSlots * kQBytes;   // [stages][K 8 KB | V 8 KB]
+  uint8_t* p_smem = kv_smem + kKvStages * kKvStageBytes;  // [2][128 x 64] bf16, K-major swizzled
   uint64_t* q_full = reinterpret_cast<uint64_t*>(p_smem + 2 * kPBytes);  // [2]
   uint64_t* q_empty = q_full + 2;            // [2]
   uint64_t* kv_full = q_empty + 2;
@@ -103,7 +105,7 @@ dca_umma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
     fence_mbar_init();
   }
   if (warp == 1) {
-    tmem_alloc(tmem_ptr, 512);
+    tmem_alloc(tmem_ptr, kTmemCols);
     tmem_relinquish();
   }
   tc_fence_before_sync();
@@ -125,8 +127,8 @@ dca_umma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
         const int32_t s0 = p.seq_offsets[item.req];
         const int32_t L = p.seq_offsets[item.req + 1] - s0;
         if (L == 0) continue;  // nobody touches a barrier for an item without keys
-        const uint32_t slot = n_work & 1;
-        if (!mbar_wait(&q_empty[slot], ((n_work >> 1) & 1) ^ 1, abort_flag, p.status, kStatusDca | 1)) { ok = false; break; }
+        const uint32_t slot = n_work % kQSlots;
+        if (!mbar_wait(&q_empty[slot], ((n_work / kQSlots) & 1) ^ 1, abort_flag, p.status, kStatusDca | 1)) { ok = false; break; }
         ++n_work;
         const int32_t sides = item.count_b > 0 ? 2 : 1;
         uint8_t* qs = q_smem + slot * 2 * kQBytes;
@@ -174,8 +176,8 @@ dca_umma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
       const uint32_t v_addr = smem_u32(kv_smem + stage * kKvStageBytes + BKV * DH * 2);
 #pragma unroll
       for (int k = 0; k < BKV / 16; ++k) {
-        // P: K-major, two 64-key blocks of 16 KB, 32 bytes per 16 keys inside a block
-        const uint64_t a_desc = smem_desc_sw128(p_addr + (k / 4) * (BQ * 128) + (k % 4) * 32, 1024, 16);
+        // P: K-major, one 64-key block (128 rows x 128 bytes), 32 bytes per 16 keys
+        const uint64_t a_desc = smem_desc_sw128(p_addr + k * 32, 1024, 16);
         // V: rows are keys (K), 128 bytes = 64 head dims (N): 16 keys = 2048 bytes further on
         const uint64_t b_desc = smem_desc_sw128(v_addr + k * 16 * 128, 1024, 16);
         umma_ss(d, a_desc, b_desc, idesc_o, (k != 0 || !first_block) ? 1u : 0u);
@@ -188,8 +190,8 @@ dca_umma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
       if (L == 0) continue;
       const int32_t sides = item.count_b > 0 ? 2 : 1;
       const int32_t nblk = (L + BKV - 1) / BKV;
-      const uint32_t slot = n_work & 1;
-      if (!mbar_wait(&q_full[slot], (n_work >> 1) & 1, abort_flag, p.status, kStatusDca | 3)) { ok = false; break; }
+      const uint32_t slot = n_work % kQSlots;
+      if (!mbar_wait(&q_full[slot], (n_work / kQSlots) & 1, abort_flag, p.status, kStatusDca | 3)) { ok = false; break; }
       ++n_work;
       // first key block: S for both sides (their S tiles were drained at the end of the previous item)
       if (!mbar_wait(&kv_full[kv_it % kKvStages], (kv_it / kKvStages) & 1, abort_flag, p.status, kStatusDca | 4)) { ok = false; break; }
@@ -321,8 +323,8 @@ dca_umma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
             h2 = __floats2bfloat162_rn(pe[2], pe[3]); w.y = *reinterpret_cast<uint32_t*>(&h2);
             h2 = __floats2bfloat162_rn(pe[4], pe[5]); w.z = *reinterpret_cast<uint32_t*>(&h2);
             h2 = __floats2bfloat162_rn(pe[6], pe[7]); w.w = *reinterpret_cast<uint32_t*>(&h2);
-            // 8 keys = one 16-byte chunk of this row inside the 64-key block c / 64
-            *reinterpret_cast<uint4*>(p_row + (c / 64) * (BQ * 128) + ((((c % 64) / 8) ^ (row & 7)) << 4)) = w;
+            // 8 keys = one 16-byte chunk of this row
+            *reinterpret_cast<uint4*>(p_row + (((c / 8) ^ (row & 7)) << 4)) = w;
           }
           l_run = l_run * alpha + sum;
           fence_proxy_async_smem();
@@ -371,7 +373,7 @@ dca_umma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
   __syncthreads();
   if (warp == 1) {
     tc_fence_after_sync();
-    tmem_dealloc(tmem_base, 512);
+    tmem_dealloc(tmem_base, kTmemCols);
   }
 }
 
@@ -426,7 +428,7 @@ rocs_status_t umma_dca(const rocs_plan* plan, int32_t n_q, int32_t H, int32_t dh
   p.n_rows = plan->N * n_q;
   p.status = status;
   ROCS_CUDA_TRY(cudaFuncSetAttribute(dca_umma_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes));
-  const int grid = std::min(items.num, sm_count_dca());
+  const int grid = std::min(items.num, 2 * sm_count_dca());  // two CTAs per SM
   dca_umma_kernel<<<grid, kThreads, kSmemBytes, stream>>>(map_q, map_k, map_v, p);
   ROCS_CUDA_TRY(cudaGetLastError());
   return ROCS_OK;
