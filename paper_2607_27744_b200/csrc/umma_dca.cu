@@ -64,6 +64,31 @@ __device__ __forceinline__ float ex2(float x) {
   return y;
 }
 
+// Packed fp32 pairs (one instruction for two lanes of arithmetic) and the three-input maximum.
+__device__ __forceinline__ uint64_t pack2(float a, float b) {
+  uint64_t r;
+  asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(a), "f"(b));
+  return r;
+}
+__device__ __forceinline__ void unpack2(uint64_t v, float& a, float& b) {
+  asm("mov.b64 {%0, %1}, %2;" : "=f"(a), "=f"(b) : "l"(v));
+}
+__device__ __forceinline__ uint64_t ffma2(uint64_t a, uint64_t b, uint64_t c) {
+  uint64_t d;
+  asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(a), "l"(b), "l"(c));
+  return d;
+}
+__device__ __forceinline__ uint64_t fadd2(uint64_t a, uint64_t b) {
+  uint64_t d;
+  asm("add.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
+  return d;
+}
+__device__ __forceinline__ float fmax3(float a, float b, float c) {
+  float d;
+  asm("max.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c));
+  return d;
+}
+
 __global__ void __launch_bounds__(kThreads, 2)
 dca_umma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
                 const __grid_constant__ CUtensorMap map_v, const DcaParams p) {
@@ -279,13 +304,13 @@ dca_umma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
             for (int e = 0; e < BKV; ++e)
               if (e >= valid) sv[e] = 0xff800000u;  // -inf: the key does not exist
           }
-          float mx4[8];
+          float mx4[4];
 #pragma unroll
-          for (int u = 0; u < 8; ++u) mx4[u] = __uint_as_float(sv[u]);
+          for (int u = 0; u < 4; ++u) mx4[u] = fmaxf(__uint_as_float(sv[2 * u]), __uint_as_float(sv[2 * u + 1]));
 #pragma unroll
-          for (int e = 8; e < BKV; ++e) mx4[e & 7] = fmaxf(mx4[e & 7], __uint_as_float(sv[e]));  // 8 short chains
-          float mx = fmaxf(fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3])),
-                           fmaxf(fmaxf(mx4[4], mx4[5]), fmaxf(mx4[6], mx4[7])));
+          for (int e = 8; e < BKV; e += 2)  // four short chains of three-input maxima
+            mx4[(e >> 1) & 3] = fmax3(mx4[(e >> 1) & 3], __uint_as_float(sv[e]), __uint_as_float(sv[e + 1]));
+          float mx = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3]));
           mx *= p.scale_log2e;
           // this row's own decision: move the reference only for a jump of more than 2^8
           const bool move = mx > m_ref + kRescaleThreshold;
@@ -310,13 +335,19 @@ dca_umma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
               tmem_st_wait();
             }
           }
-          float sum = 0.f;
+          const uint64_t c2 = pack2(p.scale_log2e, p.scale_log2e), m2 = pack2(-m_new, -m_new);
+          uint64_t sum2 = pack2(0.f, 0.f);
 #pragma unroll
           for (int c = 0; c < BKV; c += 8) {
             float pe[8];
 #pragma unroll
-            for (int e = 0; e < 8; ++e) pe[e] = ex2(fmaf(__uint_as_float(sv[c + e]), p.scale_log2e, -m_new));
-            sum += ((pe[0] + pe[1]) + (pe[2] + pe[3])) + ((pe[4] + pe[5]) + (pe[6] + pe[7]));
+            for (int e = 0; e < 8; e += 2) {
+              float x0, x1;
+              unpack2(ffma2(pack2(__uint_as_float(sv[c + e]), __uint_as_float(sv[c + e + 1])), c2, m2), x0, x1);
+              pe[e] = ex2(x0);
+              pe[e + 1] = ex2(x1);
+              sum2 = fadd2(sum2, pack2(pe[e], pe[e + 1]));
+            }
             uint4 w;
             __nv_bfloat162 h2;
             h2 = __floats2bfloat162_rn(pe[0], pe[1]); w.x = *reinterpret_cast<uint32_t*>(&h2);
@@ -326,6 +357,9 @@ dca_umma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
             // 8 keys = one 16-byte chunk of this row
             *reinterpret_cast<uint4*>(p_row + (((c / 8) ^ (row & 7)) << 4)) = w;
           }
+          float sum_lo, sum_hi;
+          unpack2(sum2, sum_lo, sum_hi);
+          const float sum = sum_lo + sum_hi;
           l_run = l_run * alpha + sum;
           fence_proxy_async_smem();
           tc_fence_before_sync();
