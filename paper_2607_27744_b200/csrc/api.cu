@@ -223,11 +223,12 @@ static rocs_status_t linear_dispatch(rocs_dtype_t dt, int64_t M, int32_t d_in, i
                                      const void* X, int64_t ld_x, const void* W, int64_t ld_w,
                                      const float* bias, const float* add, int64_t ld_add,
                                      const int32_t* row2req, int act, void* Y, int64_t ld_y,
-                                     bool out_f32, cudaStream_t stream) {
+                                     bool out_f32, cudaStream_t stream,
+                                     bool add_from_previous_launch = false) {
   if (dt == ROCS_BF16 && g_path.load() == ROCS_PATH_AUTO &&
       umma_linear_supported(M, d_in, d_out, ld_x, ld_w, ld_y, out_f32))
     return umma_linear(M, d_in, d_out, X, ld_x, W, ld_w, bias, add, ld_add, row2req, act, Y, ld_y,
-                       out_f32, stream);
+                       out_f32, stream, add_from_previous_launch);
   return simt_linear(dt, M, d_in, d_out, X, ld_x, W, ld_w, bias, add, ld_add, row2req, act, Y, ld_y,
                      out_f32, stream);
 }
@@ -266,8 +267,13 @@ rocs_status_t rocs_ikbo_linear(const rocs_plan_t* plan, rocs_dtype_t dtype, int3
     bias = nullptr;
   }
   // Candidate half with the request term gathered in the epilogue (Eq. 14, Section 4.2.1).
+  // The request half was enqueued directly in front: the candidate kernel may overlap its set-up
+  // with it (it waits for it before reading Z).  Only meaningful when both went to tensor cores.
+  const bool request_half_on_umma = Z != nullptr && dtype == ROCS_BF16 && g_path.load() == ROCS_PATH_AUTO &&
+                                    umma_linear_supported(plan->R, d_req, d_out, ld_xr, ld_wcr, d_out, true);
   return linear_dispatch(dtype, plan->N, d_cand, d_out, XC, ld_xc, W_CC, ld_wcc, bias, Z, d_out,
-                         Z ? plan->row2req : nullptr, act, Y, ld_y, /*out_f32=*/false, stream);
+                         Z ? plan->row2req : nullptr, act, Y, ld_y, /*out_f32=*/false, stream,
+                         request_half_on_umma);
 }
 
 rocs_status_t rocs_linear(rocs_dtype_t dtype, int64_t M, int32_t d_in, int32_t d_out, const void* X,

@@ -94,10 +94,13 @@ rocs_status_t simt_glm(rocs_dtype_t dt, const rocs_plan* plan, int32_t n_r, int3
 // ---- tcgen05 tensor-core kernels (bf16): umma_*.cu -------------------------------------
 bool umma_linear_supported(int64_t M, int32_t d_in, int32_t d_out, int64_t ld_x, int64_t ld_w,
                            int64_t ld_y, bool out_f32);
+// add_from_previous_launch: `add` is written by the launch directly in front of this one on the
+// stream (the request half) and nothing else this call reads is; the kernel may then overlap its
+// set-up with that launch and waits for it only before it reads `add`.
 rocs_status_t umma_linear(int64_t M, int32_t d_in, int32_t d_out, const void* X, int64_t ld_x,
                           const void* W, int64_t ld_w, const float* bias, const float* add,
                           int64_t ld_add, const int32_t* row2req, int act, void* Y, int64_t ld_y,
-                          bool out_f32, cudaStream_t stream);
+                          bool out_f32, cudaStream_t stream, bool add_from_previous_launch = false);
 // Weight-stationary variant for d_in <= 256 and bf16 output (umma_linear picks it when it applies).
 bool umma_linear_ws_supported(int64_t M, int32_t d_in, int32_t d_out, bool out_f32);
 rocs_status_t umma_linear_ws(int64_t M, int32_t d_in, int32_t d_out, const void* X, int64_t ld_x,
@@ -109,7 +112,7 @@ bool umma_linear_ws2_supported(int64_t M, int32_t d_in, int32_t d_out, bool out_
 rocs_status_t umma_linear_ws2(int64_t M, int32_t d_in, int32_t d_out, const void* X, int64_t ld_x,
                               const void* W, int64_t ld_w, const float* bias, const float* add,
                               int64_t ld_add, const int32_t* row2req, int act, void* Y, int64_t ld_y,
-                              cudaStream_t stream);
+                              cudaStream_t stream, bool add_from_previous_launch = false);
 bool umma_dca_supported(int32_t n_q, int32_t H, int32_t dh);
 rocs_status_t umma_dca(const rocs_plan* plan, int32_t n_q, int32_t H, int32_t dh, float scale,
                        const void* Q, const void* K, const void* V, const int32_t* seq_offsets,

@@ -76,6 +76,15 @@ __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, AbortF
   }
 }
 
+// ---- programmatic dependent launch ------------------------------------------------------------
+// A kernel launched with the programmatic-stream-serialization attribute may start while its
+// predecessor still runs; it must call griddep_wait() before touching anything the predecessor
+// writes.  The predecessor releases such a dependent early with griddep_launch_dependents().
+__device__ __forceinline__ void griddep_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void griddep_launch_dependents() {
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+}
+
 // ---- proxies and fences ---------------------------------------------------------------------
 __device__ __forceinline__ void fence_proxy_async_smem() {
   asm volatile("fence.proxy.async.shared::cta;" ::: "memory");

@@ -109,6 +109,10 @@ dca_umma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
   AbortFlag* abort_flag = reinterpret_cast<AbortFlag*>(tmem_ptr + 1);
 
   const int warp = threadIdx.x / 32, lane = threadIdx.x % 32;
+  if ((smem_u32(smem) & 1023u) != 0) {  // the swizzled tiles assume a 1024-byte aligned base
+    if (threadIdx.x == 0) atomicCAS(p.status, 0u, kStatusDca | 15);
+    return;
+  }
 
   if (threadIdx.x == 0) {
     for (int x = 0; x < 2; ++x) {

@@ -96,6 +96,9 @@ linear_umma_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_const
   __syncthreads();
   tc_fence_after_sync();
   const uint32_t tmem_base = *tmem_ptr;
+  // A dependent kernel launched with programmatic serialization (the candidate half behind the
+  // request half) may begin its own set-up now; it waits for this grid before it reads our output.
+  griddep_launch_dependents();
 
   if (warp == 0) {
     // ------------------------------ TMA producer ------------------------------------------
@@ -311,9 +314,10 @@ bool umma_linear_supported(int64_t M, int32_t d_in, int32_t d_out, int64_t ld_x,
 rocs_status_t umma_linear(int64_t M, int32_t d_in, int32_t d_out, const void* X, int64_t ld_x, const void* W,
                           int64_t ld_w, const float* bias, const float* add, int64_t ld_add,
                           const int32_t* row2req, int act, void* Y, int64_t ld_y, bool out_f32,
-                          cudaStream_t stream) {
+                          cudaStream_t stream, bool add_from_previous_launch) {
   if (umma_linear_ws2_supported(M, d_in, d_out, out_f32))
-    return umma_linear_ws2(M, d_in, d_out, X, ld_x, W, ld_w, bias, add, ld_add, row2req, act, Y, ld_y, stream);
+    return umma_linear_ws2(M, d_in, d_out, X, ld_x, W, ld_w, bias, add, ld_add, row2req, act, Y, ld_y, stream,
+                           add_from_previous_launch);
   if (umma_linear_ws_supported(M, d_in, d_out, out_f32))
     return umma_linear_ws(M, d_in, d_out, X, ld_x, W, ld_w, bias, add, ld_add, row2req, act, Y, ld_y, stream);
 #define ROCS_LAUNCH(BN_)                                                                                   \

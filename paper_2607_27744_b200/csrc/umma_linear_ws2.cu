@@ -46,6 +46,7 @@ struct Ws2Params {
   int64_t ld_add;
   const int32_t* row2req;
   int32_t act;
+  int32_t wait_for_previous;  // launched with programmatic serialization behind the kernel that writes `add`
   uint32_t* status;
 };
 
@@ -133,6 +134,7 @@ linear_ws2_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_consta
         }
       };
       if (has_add && group < super_tiles) fetch_req(group);
+      bool previous_done = !p.wait_for_previous;
       for (int32_t st = group; st < super_tiles && ok; st += p.groups, ++lt) {
         const int32_t m0 = st * 2 * BM + (int32_t)rank * BM;
         // X first: the MMA needs it now; the request rows are only needed by this tile's epilogue
@@ -146,6 +148,10 @@ linear_ws2_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_consta
         if (has_add) {
           const uint32_t zb = lt % kZBufs;
           if (!mbar_wait(&z_empty[zb], ((lt / kZBufs) & 1) ^ 1, abort_flag, p.status, kStatusWs2 | 5)) { ok = false; break; }
+          if (!previous_done) {  // the request half must have finished before its rows are read
+            griddep_wait();
+            previous_done = true;
+          }
           mbar_expect_tx(&z_full[zb], kZBufBytes);
 #pragma unroll
           for (int q = 0; q < 4; ++q) tma_load_2d(z_smem + (zb * 4 + q) * BN, &map_z, &z_full[zb], n0, req_next[q]);
@@ -323,7 +329,8 @@ bool umma_linear_ws2_supported(int64_t M, int32_t d_in, int32_t d_out, bool out_
 
 rocs_status_t umma_linear_ws2(int64_t M, int32_t d_in, int32_t d_out, const void* X, int64_t ld_x, const void* W,
                               int64_t ld_w, const float* bias, const float* add, int64_t ld_add,
-                              const int32_t* row2req, int act, void* Y, int64_t ld_y, cudaStream_t stream) {
+                              const int32_t* row2req, int act, void* Y, int64_t ld_y, cudaStream_t stream,
+                              bool add_from_previous_launch) {
   const int32_t k_blocks = (d_in + BK - 1) / BK;
   CUtensorMap map_x, map_w, map_z, map_y;
   if (!make_tensor_map_2d(&map_x, X, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, (uint64_t)M, (uint64_t)d_in, (uint64_t)ld_x,
@@ -350,10 +357,20 @@ rocs_status_t umma_linear_ws2(int64_t M, int32_t d_in, int32_t d_out, const void
   const int fixed = k_blocks * kWBlockBytes + kStagingBytes + kZBufs * kZBufBytes + 512 + 1024;
   p.a_stages = std::min(10, (227 * 1024 - fixed) / kAStageBytes);
   p.bias = bias; p.add = add; p.ld_add = ld_add; p.row2req = row2req; p.act = act; p.status = status;
+  p.wait_for_previous = (add_from_previous_launch && add != nullptr) ? 1 : 0;
   const int smem_bytes = fixed + p.a_stages * kAStageBytes;
   ROCS_CUDA_TRY(cudaFuncSetAttribute(linear_ws2_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_bytes));
-  linear_ws2_kernel<<<2 * p.n_slices * p.groups, kThreads, smem_bytes, stream>>>(map_x, map_w, map_z, map_y, p);
-  ROCS_CUDA_TRY(cudaGetLastError());
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(2 * p.n_slices * p.groups);
+  cfg.blockDim = dim3(kThreads);
+  cfg.dynamicSmemBytes = smem_bytes;
+  cfg.stream = stream;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = p.wait_for_previous ? 1 : 0;
+  ROCS_CUDA_TRY(cudaLaunchKernelEx(&cfg, linear_ws2_kernel, map_x, map_w, map_z, map_y, p));
   return ROCS_OK;
 }
 
