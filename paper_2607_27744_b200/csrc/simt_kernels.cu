@@ -181,11 +181,24 @@ __global__ void __launch_bounds__(256) glm_request_simt_kernel(
     for (int e = threadIdx.x; e < (n_ro + n_co) * n_r; e += blockDim.x)
       w[e] = ld_f(W, (int64_t)(e / n_r) * n + e % n_r);
   __syncthreads();
-  for (int idx = threadIdx.x; idx < n_r * n_r; idx += blockDim.x) {
-    const int a = idx / n_r, b = idx % n_r;
-    float acc = 0.f;
-    for (int e = 0; e < d; ++e) acc = fmaf(xr[a * ds + e], xr[b * ds + e], acc);
-    g[idx] = acc;
+  // four neighbouring columns of one row per thread: four independent accumulation chains
+  const int n_r4 = (n_r + 3) / 4;
+  for (int idx = threadIdx.x; idx < n_r * n_r4; idx += blockDim.x) {
+    const int a = idx / n_r4, b0 = (idx % n_r4) * 4;
+    float acc[4] = {0.f, 0.f, 0.f, 0.f};
+    const float* xa = xr + a * ds;
+    const float* xb[4];
+#pragma unroll
+    for (int u = 0; u < 4; ++u) xb[u] = xr + min(b0 + u, n_r - 1) * ds;
+#pragma unroll 4
+    for (int e = 0; e < d; ++e) {
+      const float va = xa[e];
+#pragma unroll
+      for (int u = 0; u < 4; ++u) acc[u] = fmaf(va, xb[u][e], acc[u]);
+    }
+#pragma unroll
+    for (int u = 0; u < 4; ++u)
+      if (b0 + u < n_r) g[a * n_r + b0 + u] = acc[u];
   }
   __syncthreads();
   if (YR)

@@ -164,6 +164,24 @@ def test_dca_bf16_several_query_tokens_and_scale(path):
     assert _run_dca(cfg, co, so, path=path, scale=0.2) <= tol_for("bf16")
 
 
+def test_dca_bf16_32_query_tokens_per_candidate():
+    # the paper's typical candidate-side query length (Section 4.3): four candidates fill a 128-row tile
+    co = wl.offsets_from_counts([9, 1, 30])
+    so = wl.offsets_from_counts([200, 64, 130])
+    cfg = wl.CONFIGS[3].with_(R=3, H=2, dh=64, n_q=32)
+    assert _run_dca(cfg, co, so) <= tol_for("bf16")
+
+
+def test_dca_request_side_query_group():
+    # A^R of Eq. 13 (first line) through the same kernel: one query group per request, i.e. a plan
+    # whose "candidates" are the requests themselves
+    R = 5
+    co = np.arange(R + 1, dtype=np.int32)
+    so = wl.offsets_from_counts([300, 17, 0, 128, 65])
+    cfg = wl.CONFIGS[3].with_(R=R, H=4, dh=64, n_q=16)
+    assert _run_dca(cfg, co, so) <= tol_for("bf16")
+
+
 @pytest.mark.parametrize("dh", [32, 128])
 def test_dca_bf16_other_head_dims(dh):
     co = wl.offsets_from_counts([40, 2])
