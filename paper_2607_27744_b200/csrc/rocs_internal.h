@@ -113,6 +113,11 @@ rocs_status_t umma_linear_ws2(int64_t M, int32_t d_in, int32_t d_out, const void
                               const void* W, int64_t ld_w, const float* bias, const float* add,
                               int64_t ld_add, const int32_t* row2req, int act, void* Y, int64_t ld_y,
                               cudaStream_t stream, bool add_from_previous_launch = false);
+// K-ring GEMM on CTA pairs for wide plain layers (no request term, bf16 output, many rows).
+bool umma_linear_pair_supported(int64_t M, int32_t d_in, int32_t d_out, bool out_f32, bool has_add);
+rocs_status_t umma_linear_pair(int64_t M, int32_t d_in, int32_t d_out, const void* X, int64_t ld_x,
+                               const void* W, int64_t ld_w, const float* bias, int act, void* Y,
+                               int64_t ld_y, cudaStream_t stream);
 bool umma_dca_supported(int32_t n_q, int32_t H, int32_t dh);
 rocs_status_t umma_dca(const rocs_plan* plan, int32_t n_q, int32_t H, int32_t dh, float scale,
                        const void* Q, const void* K, const void* V, const int32_t* seq_offsets,

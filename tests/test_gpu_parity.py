@@ -83,6 +83,20 @@ def test_linear_bf16_no_request_half(path):
     assert _run_linear(cfg, co, bias=True, relu=True, path=path) <= tol_for("bf16")
 
 
+@pytest.mark.parametrize("relu,bias", [(False, True), (True, False)])
+def test_plain_linear_bf16_wide_many_rows(relu, bias):
+    # M >= 2048 rows, wide K and d_out >= 256 take the CTA-pair K-ring GEMM; M is not a multiple of the
+    # 256-row super-tile and d_out = 328 leaves a ragged last column tile
+    g = np.random.default_rng(17)
+    M, d_in, d_out = 2500, 712, 328
+    X = wl.store(g.standard_normal((M, d_in), dtype=np.float32), "bf16")
+    W = wl.store(g.standard_normal((d_out, d_in), dtype=np.float32) * d_in ** -0.5, "bf16")
+    b = g.standard_normal(d_out).astype(np.float32) if bias else None
+    y = rocs.linear(to_dev(X), to_dev(W), bias=to_dev(b), relu=relu)
+    want = ref.ikbo_linear(wl.offsets_from_counts([M]), None, X, W, bias=b, relu=relu)
+    assert rel_err(to_host_f64(y), want) <= tol_for("bf16")
+
+
 def test_linear_empty_batch():
     co = np.zeros(3, np.int32)
     cfg = wl.CONFIGS[2].with_(R=2, d_req=64, d_cand=64, d_out=64)
