@@ -131,6 +131,45 @@ def test_mlp_config2_three_layers_reduced_rows():
     assert rel_err(to_host_f64(y), r) <= tol_for("bf16")
 
 
+def test_mlp_config2_full_size_sampled():
+    # the whole benchmark step (plan, split layer, two plain layers) at full size; the oracle follows
+    # the sampled candidates through all three layers in fp64
+    cfg = wl.CONFIGS[2]
+    co = wl.cand_offsets(cfg)
+    d = wl.linear_inputs(cfg, co)
+    ws = wl.mlp_weights(cfg)
+    sample = wl.stratified_sample(co, n_uniform=128, n_small_requests=0, cfg_id=2)
+    plan = _plan(co)
+    W = to_dev(d["W"])
+    h = rocs.ikbo_linear(plan, to_dev(d["XR"]), to_dev(d["XC"]), W[:, :cfg.d_req], W[:, cfg.d_req:], relu=True)
+    h = rocs.linear(h, to_dev(ws[0]), relu=True)
+    y = rocs.linear(h, to_dev(ws[1]))
+    r = ref.ikbo_linear(co, d["XR"], d["XC"], d["W"], relu=True, sample=sample)
+    one = wl.offsets_from_counts([r.shape[0]])
+    r = ref.ikbo_linear(one, None, r, wl.to_f64(ws[0]), relu=True)
+    r = ref.ikbo_linear(one, None, r, wl.to_f64(ws[1]))
+    assert rel_err(to_host_f64(y)[sample], r) <= tol_for("bf16")
+
+
+def test_isolation_config2_full_size_is_bit_exact():
+    # Eq. 1 at the size and launch configuration the benchmark times: one candidate changes, every
+    # other output row of the split layer keeps its bits
+    cfg = wl.CONFIGS[2]
+    co = wl.cand_offsets(cfg)
+    d = wl.linear_inputs(cfg, co)
+    plan = _plan(co)
+    W, XR, XC = to_dev(d["W"]), to_dev(d["XR"]), to_dev(d["XC"])
+    base = rocs.ikbo_linear(plan, XR, XC, W[:, :cfg.d_req], W[:, cfg.d_req:], relu=True)
+    j = 77_777
+    XC2 = XC.clone()
+    XC2[j] += 1.0
+    pert = rocs.ikbo_linear(plan, XR, XC2, W[:, :cfg.d_req], W[:, cfg.d_req:], relu=True)
+    same = (base.view(torch.int16) == pert.view(torch.int16)).all(dim=1)
+    assert not bool(same[j])
+    same[j] = True
+    assert bool(same.all())
+
+
 def test_linear_config2_full_size_sampled():
     cfg = wl.CONFIGS[2]
     co = wl.cand_offsets(cfg)
@@ -229,6 +268,31 @@ def test_dca_stack_config3_two_layers_reduced():
         ar = ref.dca_attention(co, so, qr.reshape(N, 1, cfg.H, cfg.dh), wl.to_f64(lay["K"]), wl.to_f64(lay["V"]))
         hr = np.concatenate([hr, ar.reshape(N, -1)], axis=1)
     assert rel_err(to_host_f64(h), hr) <= tol_for("bf16")
+
+
+def test_dca_stack_config3_full_size_sampled():
+    # two stacked DCA layers at full size: Q_l = W_Q,l h_{l-1}, A_l = DCA(Q_l, K_l, V_l), h_l = [h_{l-1}, A_l];
+    # the oracle follows a sample of candidates through both layers
+    cfg = wl.CONFIGS[3]
+    co, so = wl.cand_offsets(cfg), wl.seq_offsets(cfg)
+    d = wl.dca_stack_inputs(cfg, co, so)
+    plan = _plan(co)
+    N = int(co[-1])
+    sample = wl.stratified_sample(co, n_uniform=24, n_small_requests=0, cfg_id=3)[::4]
+    h = to_dev(d["XC"])
+    hr = wl.to_f64(d["XC"])[sample]
+    one = wl.offsets_from_counts([sample.size])
+    for lay in d["layers"]:
+        q = rocs.linear(h, to_dev(lay["WQ"]))
+        a = rocs.dca_attention(plan, q.view(N, 1, cfg.H, cfg.dh), to_dev(lay["K"]), to_dev(lay["V"]), to_dev(so))
+        h = torch.cat([h, a.view(N, -1)], dim=1).contiguous()
+        qr = ref.ikbo_linear(one, None, hr, wl.to_f64(lay["WQ"]))
+        # the oracle attends the sampled rows against their own requests: scatter them into a full-size Q
+        Qf = np.zeros((N, 1, cfg.H, cfg.dh))
+        Qf[sample] = qr.reshape(-1, 1, cfg.H, cfg.dh)
+        ar = ref.dca_attention(co, so, Qf, wl.to_f64(lay["K"]), wl.to_f64(lay["V"]), sample=sample)
+        hr = np.concatenate([hr, ar.reshape(sample.size, -1)], axis=1)
+    assert rel_err(to_host_f64(h)[sample], hr) <= tol_for("bf16")
 
 
 def test_dca_config3_full_size_sampled():
