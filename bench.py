@@ -335,28 +335,53 @@ def run_rocs(args):
         extra = bench_other_ops(torch, rocs, peaks, dev, time_call, args.extra.split(","))
 
     # ---- end to end from pinned host buffers ------------------------------------------------
+    # Every step copies its inputs from pinned host memory and reads its scores back.  The three
+    # phases of consecutive steps are pipelined on three streams (copy-in of step i+1 and copy-out of
+    # step i-1 run beside the kernels of step i), with two sets of device input buffers and of host
+    # output buffers; every step still moves all of its bytes inside the timed region.
     XR_h, XC_h, co_h = pinned(data["lin"]["XR"]), pinned(data["lin"]["XC"]), pinned(co)
-    y_h = torch.empty((N, 256), dtype=torch.bfloat16).pin_memory()
-    XR_d, XC_d, co_d = torch.empty_like(XR_sets[0]), torch.empty_like(XC_sets[0]), torch.empty_like(co_dev)
+    y_h = [torch.empty((N, 256), dtype=torch.bfloat16).pin_memory() for _ in range(2)]
+    in_d = [(torch.empty_like(XR_sets[0]), torch.empty_like(XC_sets[0]), torch.empty_like(co_dev)) for _ in range(2)]
+    s_in, s_cmp, s_out = torch.cuda.Stream(), torch.cuda.Stream(), torch.cuda.Stream()
 
-    def e2e_step(i):
-        XR_d.copy_(XR_h, non_blocking=True)
-        XC_d.copy_(XC_h, non_blocking=True)
-        co_d.copy_(co_h, non_blocking=True)
-        out = step(i, XR_d, XC_d, co_d)
-        y_h.copy_(out, non_blocking=True)
+    def e2e_run(n_steps):
+        in_done = [None, None]
+        cmp_done = [None, None]     # kernels of the step that last used input set / output y[s]
+        out_done = [None, None]
+        for i in range(n_steps):
+            b = i % 2
+            with torch.cuda.stream(s_in):
+                if cmp_done[b] is not None:
+                    s_in.wait_event(cmp_done[b])          # input set b is free again
+                in_d[b][0].copy_(XR_h, non_blocking=True)
+                in_d[b][1].copy_(XC_h, non_blocking=True)
+                in_d[b][2].copy_(co_h, non_blocking=True)
+                in_done[b] = torch.cuda.Event()
+                in_done[b].record(s_in)
+            with torch.cuda.stream(s_cmp):
+                s_cmp.wait_event(in_done[b])
+                if out_done[b] is not None:
+                    s_cmp.wait_event(out_done[b])        # y[s] of this parity has been read back
+                out = step(b, in_d[b][0], in_d[b][1], in_d[b][2])
+                cmp_done[b] = torch.cuda.Event()
+                cmp_done[b].record(s_cmp)
+            with torch.cuda.stream(s_out):
+                s_out.wait_event(cmp_done[b])
+                y_h[b].copy_(out, non_blocking=True)
+                out_done[b] = torch.cuda.Event()
+                out_done[b].record(s_out)
+        for st in (s_in, s_cmp, s_out):
+            torch.cuda.current_stream().wait_stream(st)
 
-    for i in range(args.warmup):
-        e2e_step(i)
+    e2e_run(args.warmup)
     barrier()
     e0.record()
-    for i in range(args.steps):
-        e2e_step(i)
+    e2e_run(args.steps)
     e1.record()
     barrier()
     e2e_ms = max_over_ranks(e0.elapsed_time(e1)) / args.steps
     h2d = XR_h.numel() * 2 + XC_h.numel() * 2 + co_h.numel() * 4
-    d2h = y_h.numel() * 2
+    d2h = y_h[0].numel() * 2
 
     if rank != 0:
         return
