@@ -109,7 +109,7 @@ linear_pair_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_const
     }
   } else if (warp == 1) {
     // ------------------------------ MMA issuer (leader CTA only) ---------------------------
-    if (rank == 0) {
+    if (rank == 0 && lane == 0) {
       constexpr uint32_t idesc = umma_idesc_bf16(2 * BM, BN, false, false);
       uint32_t it = 0, lt = 0;
       bool ok = true;
@@ -122,21 +122,17 @@ linear_pair_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_const
           const int s = it % kStages;
           if (!mbar_wait(&full[s], (it / kStages) & 1, abort_flag, p.status, kStatusPair | 3)) { ok = false; break; }
           tc_fence_after_sync();
-          if (lane == 0) {
-            const uint32_t st = smem_u32(smem + s * kStageBytes);
-            const uint64_t a_desc = smem_desc_sw128(st, 1024, 16);
-            const uint64_t b_desc = smem_desc_sw128(st + kABytes, 1024, 16);
+          const uint32_t st = smem_u32(smem + s * kStageBytes);
+          const uint64_t a_desc = smem_desc_sw128(st, 1024, 16);
+          const uint64_t b_desc = smem_desc_sw128(st + kABytes, 1024, 16);
 #pragma unroll
-            for (int k = 0; k < BK / 16; ++k)
-              umma_ss_pair(d_tmem, a_desc + 2 * k, b_desc + 2 * k, idesc, (kb | k) != 0 ? 1u : 0u);
-            umma_commit_pair(&empty[s], 3);
-          }
-          __syncwarp();
+          for (int k = 0; k < BK / 16; ++k)
+            umma_ss_pair(d_tmem, a_desc + 2 * k, b_desc + 2 * k, idesc, (kb | k) != 0 ? 1u : 0u);
+          umma_commit_pair(&empty[s], 3);
         }
-        if (ok && lane == 0) umma_commit_pair(&tmem_full[acc], 3);
-        __syncwarp();
+        if (ok) umma_commit_pair(&tmem_full[acc], 3);
       }
-      if (!ok && lane == 0) {
+      if (!ok) {
         umma_commit_pair(drain, 1);
         const uint64_t t0 = globaltimer_ns();
         while (!mbar_try_wait(drain, 0) && globaltimer_ns() - t0 < kWaitLimitNs) {}
