@@ -157,7 +157,7 @@ dca_umma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
         const int32_t L = p.seq_offsets[item.req + 1] - s0;
         if (L == 0) continue;  // nobody touches a barrier for an item without keys
         const uint32_t slot = n_work % kQSlots;
-        if (!mbar_wait(&q_empty[slot], ((n_work / kQSlots) & 1) ^ 1, abort_flag, p.status, kStatusDca | 1)) { ok = false; break; }
+        if (!mbar_wait_paced(&q_empty[slot], ((n_work / kQSlots) & 1) ^ 1, abort_flag, p.status, kStatusDca | 1)) { ok = false; break; }
         ++n_work;
         const int32_t sides = item.count_b > 0 ? 2 : 1;
         uint8_t* qs = q_smem + slot * 2 * kQBytes;
@@ -167,7 +167,7 @@ dca_umma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
         const int32_t nblk = (L + BKV - 1) / BKV;
         for (int32_t j = 0; j < nblk; ++j, ++kv_it) {
           const int s = kv_it % kKvStages;
-          if (!mbar_wait(&kv_empty[s], ((kv_it / kKvStages) & 1) ^ 1, abort_flag, p.status, kStatusDca | 2)) { ok = false; break; }
+          if (!mbar_wait_paced(&kv_empty[s], ((kv_it / kKvStages) & 1) ^ 1, abort_flag, p.status, kStatusDca | 2)) { ok = false; break; }
           uint8_t* st = kv_smem + s * kKvStageBytes;
           mbar_expect_tx(&kv_full[s], kKvStageBytes);
           tma_load_2d(st, &map_k, &kv_full[s], item.head * DH, s0 + j * BKV);
@@ -220,10 +220,10 @@ dca_umma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
       const int32_t sides = item.count_b > 0 ? 2 : 1;
       const int32_t nblk = (L + BKV - 1) / BKV;
       const uint32_t slot = n_work % kQSlots;
-      if (!mbar_wait(&q_full[slot], (n_work / kQSlots) & 1, abort_flag, p.status, kStatusDca | 3)) { ok = false; break; }
+      if (!mbar_wait_paced(&q_full[slot], (n_work / kQSlots) & 1, abort_flag, p.status, kStatusDca | 3)) { ok = false; break; }
       ++n_work;
       // first key block: S for both sides (their S tiles were drained at the end of the previous item)
-      if (!mbar_wait(&kv_full[kv_it % kKvStages], (kv_it / kKvStages) & 1, abort_flag, p.status, kStatusDca | 4)) { ok = false; break; }
+      if (!mbar_wait_paced(&kv_full[kv_it % kKvStages], (kv_it / kKvStages) & 1, abort_flag, p.status, kStatusDca | 4)) { ok = false; break; }
       tc_fence_after_sync();
       if (lane == 0) {
         for (int x = 0; x < sides; ++x) issue_s(x, kv_it % kKvStages, slot);
@@ -234,10 +234,10 @@ dca_umma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
         const int stage = kv_it % kKvStages;
         const int next_stage = (kv_it + 1) % kKvStages;
         if (j + 1 < nblk) {
-          if (!mbar_wait(&kv_full[next_stage], ((kv_it + 1) / kKvStages) & 1, abort_flag, p.status, kStatusDca | 5)) { ok = false; break; }
+          if (!mbar_wait_paced(&kv_full[next_stage], ((kv_it + 1) / kKvStages) & 1, abort_flag, p.status, kStatusDca | 5)) { ok = false; break; }
           // S_{j+1} as soon as the side has pulled S_j into registers
           for (int x = 0; x < sides; ++x) {
-            if (!mbar_wait(&s_empty[x], cnt_se[x] & 1, abort_flag, p.status, kStatusDca | 11)) { ok = false; break; }
+            if (!mbar_wait_paced(&s_empty[x], cnt_se[x] & 1, abort_flag, p.status, kStatusDca | 11)) { ok = false; break; }
             ++cnt_se[x];
             tc_fence_after_sync();
             if (lane == 0) issue_s(x, next_stage, slot);
@@ -249,14 +249,14 @@ dca_umma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
         } else {
           // keep the s_empty phases in step: the sides still signal after reading the last S
           for (int x = 0; x < sides; ++x) {
-            if (!mbar_wait(&s_empty[x], cnt_se[x] & 1, abort_flag, p.status, kStatusDca | 12)) { ok = false; break; }
+            if (!mbar_wait_paced(&s_empty[x], cnt_se[x] & 1, abort_flag, p.status, kStatusDca | 12)) { ok = false; break; }
             ++cnt_se[x];
           }
           if (!ok) break;
         }
         for (int x = 0; x < sides; ++x) {
           // P_j of this side is in shared memory (and O has been rescaled if it had to be)
-          if (!mbar_wait(&p_full[x], cnt_p[x] & 1, abort_flag, p.status, kStatusDca | 6)) { ok = false; break; }
+          if (!mbar_wait_paced(&p_full[x], cnt_p[x] & 1, abort_flag, p.status, kStatusDca | 6)) { ok = false; break; }
           ++cnt_p[x];
           tc_fence_after_sync();
           if (lane == 0) issue_pv(x, stage, j == 0);
@@ -293,7 +293,7 @@ dca_umma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
         const int32_t nblk = (L + BKV - 1) / BKV;
         for (int32_t j = 0; j < nblk; ++j) {
           const int32_t valid = min(BKV, L - j * BKV);  // keys of this block that exist
-          if (!mbar_wait(&s_full[side], cnt_s & 1, abort_flag, p.status, kStatusDca | 7)) { aborted = true; break; }
+          if (!mbar_wait_paced(&s_full[side], cnt_s & 1, abort_flag, p.status, kStatusDca | 7)) { aborted = true; break; }
           ++cnt_s;
           tc_fence_after_sync();
           uint32_t sv[BKV];
@@ -323,7 +323,7 @@ dca_umma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
           m_ref = m_new;
           if (j > 0) {
             // P V of the previous block is complete: O is stable and P's buffer may be rewritten
-            if (!mbar_wait(&o_full[side], cnt_o & 1, abort_flag, p.status, kStatusDca | 8)) { aborted = true; break; }
+            if (!mbar_wait_paced(&o_full[side], cnt_o & 1, abort_flag, p.status, kStatusDca | 8)) { aborted = true; break; }
             ++cnt_o;
             tc_fence_after_sync();
             if (__any_sync(0xffffffffu, move)) {
@@ -371,7 +371,7 @@ dca_umma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
           if (lane == 0) mbar_arrive(&p_full[side]);
         }
         if (!aborted) {
-          if (!mbar_wait(&o_full[side], cnt_o & 1, abort_flag, p.status, kStatusDca | 9)) {
+          if (!mbar_wait_paced(&o_full[side], cnt_o & 1, abort_flag, p.status, kStatusDca | 9)) {
             aborted = true;
           } else {
             ++cnt_o;
