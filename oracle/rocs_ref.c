@@ -374,3 +374,105 @@ int rocs_ref_glm_interaction_decomposed(int dtype, int32_t R, int64_t N, const i
   free(zr);
   return 0;
 }
+
+/* ------------------------------------------------------------------------- *
+ * GLM factorization machine followed by a projection of its column axis
+ * (Eq. 9-10, then the k-column compression an FM block applies to its
+ * n x n interaction matrix; k is the "compression dimension" of the Wukong
+ * row of the hyper-parameter table in the appendix).  The paper prints no
+ * formula for the projection; the reading taken here is  F = G P  with a
+ * learned P in R^{n x k}, G the masked interaction matrix of Eq. 9-10.
+ * Materialised form: X = [X^R[m_i] ; X^C[i]] per candidate, G = X X^T with
+ * G[0:n_r, n_r:] = 0, F = G P.  F_out [rows, n, k] fp64: first n_r rows are
+ * the request side, the last n_c rows the candidate side.
+ * ------------------------------------------------------------------------- */
+int rocs_ref_glm_fm_projection(int dtype, int32_t R, int64_t N, const int32_t *cand_offsets,
+                               int32_t n_r, int32_t n_c, int32_t d, int32_t k, const void *XR,
+                               const void *XC, const void *P, const int64_t *sample, int64_t n_sample,
+                               double *F_out) {
+  int32_t *m = materialise_index_map(R, N, cand_offsets);
+  if (!m) return -1;
+  const int64_t rows = sample ? n_sample : N;
+  const int32_t n = n_r + n_c;
+#pragma omp parallel
+  {
+    double *X = (double *)malloc(sizeof(double) * (size_t)n * d);
+    double *G = (double *)malloc(sizeof(double) * (size_t)n * n);
+#pragma omp for schedule(dynamic, 16)
+    for (int64_t s = 0; s < rows; ++s) {
+      const int64_t i = pick(sample, s);
+      const int32_t r = m[i];
+      for (int32_t a = 0; a < n_r; ++a)
+        for (int32_t e = 0; e < d; ++e) X[a * d + e] = load_as_f64(XR, dtype, ((int64_t)r * n_r + a) * d + e);
+      for (int32_t a = 0; a < n_c; ++a)
+        for (int32_t e = 0; e < d; ++e) X[(n_r + a) * d + e] = load_as_f64(XC, dtype, (i * n_c + a) * d + e);
+      for (int32_t a = 0; a < n; ++a)
+        for (int32_t b = 0; b < n; ++b) {
+          double acc = 0.0;
+          for (int32_t e = 0; e < d; ++e) acc += X[a * d + e] * X[b * d + e];
+          G[a * n + b] = acc;
+        }
+      for (int32_t a = 0; a < n_r; ++a)
+        for (int32_t b = n_r; b < n; ++b) G[a * n + b] = 0.0;
+      for (int32_t a = 0; a < n; ++a)
+        for (int32_t c = 0; c < k; ++c) {
+          double acc = 0.0;
+          for (int32_t b = 0; b < n; ++b) acc += G[a * n + b] * load_as_f64(P, dtype, (int64_t)b * k + c);
+          F_out[(s * n + a) * k + c] = acc;
+        }
+    }
+    free(X);
+    free(G);
+  }
+  free(m);
+  return 0;
+}
+
+/* Request-once form of the same operator (Section 4.1 applied to F = G P):
+ *   T[r]  = X^R_r^T P_R                 [R, d, k]     (P_R = P[0:n_r], P_C = P[n_r:])
+ *   FR[r] = X^R_r T[r]                  [R, n_r, k]
+ *   FC[i] = X^C_i (T[m_i] + X^C_i^T P_C)   [N, n_c, k]
+ * Only for the both-forms-agree test. */
+int rocs_ref_glm_fm_projection_decomposed(int dtype, int32_t R, int64_t N, const int32_t *cand_offsets,
+                                          int32_t n_r, int32_t n_c, int32_t d, int32_t k, const void *XR,
+                                          const void *XC, const void *P, double *FR, double *FC) {
+  (void)N;
+  double *T = (double *)malloc(sizeof(double) * (size_t)d * k);
+  double *H = (double *)malloc(sizeof(double) * (size_t)d * k);
+  if (!T || !H) return -1;
+  for (int32_t r = 0; r < R; ++r) {
+    for (int32_t e = 0; e < d; ++e)
+      for (int32_t c = 0; c < k; ++c) {
+        double acc = 0.0;
+        for (int32_t a = 0; a < n_r; ++a)
+          acc += load_as_f64(XR, dtype, ((int64_t)r * n_r + a) * d + e) * load_as_f64(P, dtype, (int64_t)a * k + c);
+        T[e * k + c] = acc;
+      }
+    if (FR)
+      for (int32_t a = 0; a < n_r; ++a)
+        for (int32_t c = 0; c < k; ++c) {
+          double acc = 0.0;
+          for (int32_t e = 0; e < d; ++e) acc += load_as_f64(XR, dtype, ((int64_t)r * n_r + a) * d + e) * T[e * k + c];
+          FR[((int64_t)r * n_r + a) * k + c] = acc;
+        }
+    for (int64_t i = cand_offsets[r]; i < cand_offsets[r + 1]; ++i) {
+      for (int32_t e = 0; e < d; ++e)
+        for (int32_t c = 0; c < k; ++c) {
+          double acc = T[e * k + c];
+          for (int32_t a = 0; a < n_c; ++a)
+            acc += load_as_f64(XC, dtype, (i * n_c + a) * d + e) * load_as_f64(P, dtype, (int64_t)(n_r + a) * k + c);
+          H[e * k + c] = acc;
+        }
+      if (FC)
+        for (int32_t a = 0; a < n_c; ++a)
+          for (int32_t c = 0; c < k; ++c) {
+            double acc = 0.0;
+            for (int32_t e = 0; e < d; ++e) acc += load_as_f64(XC, dtype, (i * n_c + a) * d + e) * H[e * k + c];
+            FC[(i * n_c + a) * k + c] = acc;
+          }
+    }
+  }
+  free(T);
+  free(H);
+  return 0;
+}

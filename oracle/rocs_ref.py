@@ -201,3 +201,43 @@ def glm_interaction_decomposed(cand_offsets, XR, XC, W=None, n_ro=0, n_co=0):
         _ptr(YR), _ptr(YC), _ptr(OR), _ptr(OC))
     assert rc == 0
     return YR, YC, OR, OC
+
+
+def glm_fm_projection(cand_offsets, XR, XC, P, sample=None):
+    """Eq. 9-10 on the materialised X = [X^R[m_i]; X^C[i]], then F = G P (P [n_r + n_c, k]).
+
+    Returns F [rows, n, k]: first n_r rows request side, last n_c rows candidate side."""
+    co = _offsets(cand_offsets)
+    R, N = co.size - 1, int(co[-1])
+    XR, XC, P = _c(XR), _c(XC), _c(P)
+    n_r, d = XR.shape[1], XR.shape[2]
+    n_c = XC.shape[1]
+    n = n_r + n_c
+    assert XC.shape[0] == N and XC.shape[2] == d and P.shape[0] == n
+    k = P.shape[1]
+    dt = _same_dtype(XR, XC, P)
+    s, ns = _sample(sample)
+    rows = ns if s is not None else N
+    F = np.empty((rows, n, k), np.float64)
+    rc = _load().rocs_ref_glm_fm_projection(
+        dt, R, ctypes.c_int64(N), _ptr(co), n_r, n_c, d, k, _ptr(XR), _ptr(XC), _ptr(P),
+        _ptr(s), ctypes.c_int64(ns), _ptr(F))
+    assert rc == 0
+    return F
+
+
+def glm_fm_projection_decomposed(cand_offsets, XR, XC, P):
+    """Request-once form: returns (FR [R, n_r, k], FC [N, n_c, k])."""
+    co = _offsets(cand_offsets)
+    R, N = co.size - 1, int(co[-1])
+    XR, XC, P = _c(XR), _c(XC), _c(P)
+    n_r, d = XR.shape[1], XR.shape[2]
+    n_c = XC.shape[1]
+    k = P.shape[1]
+    dt = _same_dtype(XR, XC, P)
+    FR = np.empty((R, n_r, k), np.float64)
+    FC = np.empty((N, n_c, k), np.float64)
+    rc = _load().rocs_ref_glm_fm_projection_decomposed(
+        dt, R, ctypes.c_int64(N), _ptr(co), n_r, n_c, d, k, _ptr(XR), _ptr(XC), _ptr(P), _ptr(FR), _ptr(FC))
+    assert rc == 0
+    return FR, FC

@@ -230,6 +230,12 @@ def glm_inputs(cfg: Config, co: Optional[np.ndarray] = None):
     )
 
 
+def fm_projection_weight(cfg: Config, k: int) -> np.ndarray:
+    """Projection P [n_r + n_c, k] of the interaction matrix's column axis, N(0, 1/n)."""
+    n = cfg.n_r + cfg.n_c
+    return normal((n, k), cfg.cfg_id, 53, cfg.dtype, std=n ** -0.5)
+
+
 def stratified_sample(co: np.ndarray, n_uniform: int = 256, n_small_requests: int = 8,
                       whole_largest: bool = False, seed_stream: int = 90, cfg_id: int = 0) -> np.ndarray:
     """Candidate indices for sampled checks at full size: first and last candidate of every
