@@ -208,6 +208,26 @@ rocs_status_t rocs_glm_interaction(const rocs_plan_t* plan, rocs_dtype_t dtype, 
                                    size_t workspace_bytes, void* stream);
 
 /*
+ * GLM factorization machine for two groups (Eq. 9-10) followed by a projection of the
+ * interaction matrix's column axis to k columns (the compression an FM block applies to its
+ * n x n output; the paper names the dimension k but prints no formula, so this entry point
+ * takes the reading F = G P).  With n = n_r + n_c, P = [P_R; P_C] in R^{n x k}:
+ *     FR[r] = X^R_r X^R_r^T P_R                                      [R, n_r, k]  once per request
+ *     FC[i] = X^C_i X^R_{m_i}^T P_R + X^C_i X^C_i^T P_C              [N, n_c, k]
+ * evaluated as FC[i] = X^C_i (T[m_i] + X^C_i^T P_C) with T[r] = X^R_r^T P_R formed once per
+ * request (fp32, in `workspace`): no request tensor is replicated per candidate.
+ *   XR [R, n_r, d] dense;  XC [N, n_c, d] dense;  P [n_r + n_c, k] dense row-major
+ *   FR, FC: either may be NULL (not written);  d * sizeof(element) multiple of 16
+ *   workspace >= rocs_glm_fm_projection_workspace(...) bytes, 256-byte aligned
+ * Errors: INVALID_ARG, ALIGNMENT, WORKSPACE, UNSUPPORTED, CUDA.
+ */
+size_t rocs_glm_fm_projection_workspace(const rocs_plan_t* plan, int32_t d, int32_t k);
+rocs_status_t rocs_glm_fm_projection(const rocs_plan_t* plan, rocs_dtype_t dtype, int32_t n_r,
+                                     int32_t n_c, int32_t d, int32_t k, const void* XR,
+                                     const void* XC, const void* P, void* FR, void* FC,
+                                     void* workspace, size_t workspace_bytes, void* stream);
+
+/*
  * Device-side status of the tensor-core kernels.  Their barrier waits are bounded; a wait
  * that expires records a code in a device word instead of spinning forever and the kernel
  * returns.  This call synchronises the device, reads the word, clears it and returns

@@ -29,6 +29,7 @@ EXPORTS = [
     "rocs_status_string", "rocs_padded_ld", "rocs_set_path", "rocs_plan_create", "rocs_plan_destroy",
     "rocs_ikbo_linear_workspace", "rocs_ikbo_linear", "rocs_linear", "rocs_dca_attention_workspace",
     "rocs_dca_attention", "rocs_glm_interaction_workspace", "rocs_glm_interaction",
+    "rocs_glm_fm_projection_workspace", "rocs_glm_fm_projection",
     "rocs_last_device_status", "rocs_ikbo_linear_static", "rocs_ikbo_linear_static_max_z_elems",
     "rocs_ikbo_linear_static_max_candidates",
 ]
@@ -69,6 +70,9 @@ def lib() -> ctypes.CDLL:
         L.rocs_glm_interaction_workspace.argtypes = [vp, i32, i32, i32]
         L.rocs_glm_interaction.argtypes = [vp, ctypes.c_int, i32, i32, i32, vp, vp, vp, i32, i32, vp, vp, vp, vp,
                                            vp, sz, vp]
+        L.rocs_glm_fm_projection_workspace.restype = sz
+        L.rocs_glm_fm_projection_workspace.argtypes = [vp, i32, i32]
+        L.rocs_glm_fm_projection.argtypes = [vp, ctypes.c_int, i32, i32, i32, i32, vp, vp, vp, vp, vp, vp, sz, vp]
         L.rocs_last_device_status.argtypes = [ctypes.POINTER(ctypes.c_uint32)]
         L.rocs_ikbo_linear_static_max_z_elems.restype = sz
         L.rocs_ikbo_linear_static_max_candidates.restype = sz
@@ -250,6 +254,35 @@ def glm_interaction(plan: Plan, XR: torch.Tensor, XC: torch.Tensor, W: Optional[
         _p(outs.get("YR")), _p(outs.get("YC")), _p(outs.get("OR")), _p(outs.get("OC")),
         _p(workspace), workspace.numel() if workspace is not None else 0, _stream())
     _check(code, "rocs_glm_interaction")
+    return outs
+
+
+def glm_fm_projection_workspace(plan: Plan, d: int, k: int) -> int:
+    return int(lib().rocs_glm_fm_projection_workspace(plan.handle, d, k))
+
+
+def glm_fm_projection(plan: Plan, XR: torch.Tensor, XC: torch.Tensor, P: torch.Tensor,
+                      want_request_side: bool = True, workspace: Optional[torch.Tensor] = None,
+                      outs: Optional[dict] = None) -> dict:
+    """GLM factorization machine (Eq. 9-10) projected to k columns, F = G P with P [n_r + n_c, k].
+    Returns a dict with FC [N, n_c, k] and, if requested, FR [R, n_r, k]."""
+    R, n_r, d = XR.shape
+    N, n_c, _ = XC.shape
+    k = P.shape[1]
+    assert R == plan.R and N == plan.N and XR.is_contiguous() and XC.is_contiguous()
+    assert P.shape[0] == n_r + n_c and P.is_contiguous() and P.dtype == XC.dtype
+    dev, dt = XC.device, XC.dtype
+    outs = dict(outs or {})
+    if want_request_side:
+        outs.setdefault("FR", torch.empty((R, n_r, k), dtype=dt, device=dev))
+    outs.setdefault("FC", torch.empty((N, n_c, k), dtype=dt, device=dev))
+    need = glm_fm_projection_workspace(plan, d, k)
+    if workspace is None:
+        workspace = torch.empty(need, dtype=torch.uint8, device=dev)
+    code = lib().rocs_glm_fm_projection(
+        plan.handle, _dtype_code(XC), n_r, n_c, d, k, _p(XR), _p(XC), _p(P), _p(outs.get("FR")), _p(outs.get("FC")),
+        _p(workspace), workspace.numel(), _stream())
+    _check(code, "rocs_glm_fm_projection")
     return outs
 
 

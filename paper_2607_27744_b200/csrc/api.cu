@@ -349,6 +349,27 @@ rocs_status_t rocs_glm_interaction(const rocs_plan_t* plan, rocs_dtype_t dtype, 
   return simt_glm(dtype, plan, n_r, n_c, d, XR, XC, W, n_ro, n_co, YR, YC, OR_, OC, zr, stream);
 }
 
+size_t rocs_glm_fm_projection_workspace(const rocs_plan_t* plan, int32_t d, int32_t k) {
+  if (!plan || d <= 0 || k <= 0) return 0;
+  return round_up((size_t)std::max(plan->R, 1) * (size_t)k * (size_t)d * sizeof(float), 256);
+}
+
+rocs_status_t rocs_glm_fm_projection(const rocs_plan_t* plan, rocs_dtype_t dtype, int32_t n_r, int32_t n_c,
+                                     int32_t d, int32_t k, const void* XR, const void* XC, const void* P,
+                                     void* FR, void* FC, void* workspace, size_t workspace_bytes, void* stream_) {
+  if (!plan || (dtype != ROCS_BF16 && dtype != ROCS_F32)) return ROCS_ERR_INVALID_ARG;
+  if (n_r <= 0 || n_c <= 0 || d <= 0 || k <= 0 || !P) return ROCS_ERR_INVALID_ARG;
+  if ((plan->R > 0 && !XR) || (plan->N > 0 && FC && !XC)) return ROCS_ERR_INVALID_ARG;
+  if (!aligned16(XR) || !aligned16(XC) || !aligned16(P) || !aligned16(FR) || !aligned16(FC) ||
+      ((int64_t)d * (int64_t)elem_size(dtype)) % 16 != 0)
+    return ROCS_ERR_ALIGNMENT;
+  const size_t need = rocs_glm_fm_projection_workspace(plan, d, k);
+  if (!workspace || workspace_bytes < need || (reinterpret_cast<uintptr_t>(workspace) & 255u))
+    return ROCS_ERR_WORKSPACE;
+  return fm_projection(dtype, plan, n_r, n_c, d, k, XR, XC, P, FR, FC, (float*)workspace,
+                       g_path.load() == ROCS_PATH_AUTO, (cudaStream_t)stream_);
+}
+
 rocs_status_t rocs_last_device_status(uint32_t* detail_host) {
   uint32_t* word = device_status_word();
   if (!word) return ROCS_ERR_CUDA;

@@ -1,0 +1,363 @@
+// Projected factorization machine for two groups: F = G P, G the masked interaction matrix of
+// Eq. 9-10 and P [n_r + n_c, k] a projection of its column axis (the compression dimension k of an
+// FM block).  With P = [P_R; P_C] the in-kernel-broadcast form (Section 4.1) is
+//     T[r]  = X^R_r^T P_R                       [d, k]   once per request, fp32, in the workspace
+//     FR[r] = X^R_r T[r]                        [n_r, k] once per request
+//     FC[i] = X^C_i (T[m_i] + X^C_i^T P_C)      [n_c, k] per candidate
+// so a candidate reads its own 2 n_c d bytes and nothing of the request but the d x k block T,
+// which stays in registers while consecutive candidates belong to the same request.
+//
+// The candidate side is bound by HBM (about 30 flop per byte): the bf16 kernel streams candidate
+// tiles through a TMA ring and gives every warp one candidate at a time, whose two small products
+// (16 x d x 16 each) run on mma.sync m16n8k16 straight out of the swizzled tile:
+//   step 1   H^T = T^T + P_C^T X^C_i    accumulators start at T^T (fp32); X^C_i is the K x N
+//                                       operand, read with ldmatrix.trans
+//   step 2   FC_i = X^C_i H             H rounded to bf16 once: the accumulator layout of step 1
+//                                       is the B-operand layout of step 2, so it never leaves
+//                                       registers; X^C_i is the M x K operand, read with ldmatrix
+// A general kernel (any shape, fp32 or bf16 storage, fp32 FMA) covers everything else.
+#include <algorithm>
+
+#include "rocs_internal.h"
+#include "sm100_ptx.cuh"
+
+namespace rocs {
+namespace {
+
+using namespace ptx;
+
+__device__ __forceinline__ float ld_f(const float* p, int64_t i) { return p[i]; }
+__device__ __forceinline__ float ld_f(const __nv_bfloat16* p, int64_t i) { return __bfloat162float(p[i]); }
+__device__ __forceinline__ void st_f(float* p, int64_t i, float v) { p[i] = v; }
+__device__ __forceinline__ void st_f(__nv_bfloat16* p, int64_t i, float v) { p[i] = __float2bfloat16_rn(v); }
+
+// ---------------------------------------------------------------------------------------------
+// Request side, one block per request:  TT[r] = P_R^T X^R_r  ([k, d] fp32, the transpose of T)
+// and FR[r] = X^R_r T[r].
+// ---------------------------------------------------------------------------------------------
+template <typename T>
+__global__ void __launch_bounds__(256) fm_request_kernel(int32_t n_r, int32_t d, int32_t k, const T* __restrict__ XR,
+                                                         const T* __restrict__ P, float* __restrict__ TT,
+                                                         T* __restrict__ FR) {
+  extern __shared__ float sm[];
+  const int32_t ds = d + 1;           // padded row stride: rows land in different banks
+  float* xr = sm;                     // [n_r, d + 1]
+  float* tt = xr + (size_t)n_r * ds;  // [k, d + 1]
+  float* pr = tt + (size_t)k * ds;    // [n_r, k]
+  const int32_t r = blockIdx.x;
+  for (int e = threadIdx.x; e < n_r * d; e += blockDim.x) xr[(e / d) * ds + e % d] = ld_f(XR, (int64_t)r * n_r * d + e);
+  for (int e = threadIdx.x; e < n_r * k; e += blockDim.x) pr[e] = ld_f(P, e);
+  __syncthreads();
+  for (int idx = threadIdx.x; idx < k * d; idx += blockDim.x) {
+    const int c = idx / d, e = idx % d;
+    float acc = 0.f;
+    for (int a = 0; a < n_r; ++a) acc = fmaf(pr[a * k + c], xr[a * ds + e], acc);
+    tt[c * ds + e] = acc;
+    TT[((int64_t)r * k + c) * d + e] = acc;
+  }
+  if (!FR) return;
+  __syncthreads();
+  for (int idx = threadIdx.x; idx < n_r * k; idx += blockDim.x) {
+    const int a = idx / k, c = idx % k;
+    float acc = 0.f;
+    for (int e = 0; e < d; ++e) acc = fmaf(xr[a * ds + e], tt[c * ds + e], acc);
+    st_f(FR, ((int64_t)r * n_r + a) * k + c, acc);
+  }
+}
+
+// ---------------------------------------------------------------------------------------------
+// Candidate side, general kernel: one block per candidate.
+// ---------------------------------------------------------------------------------------------
+template <typename T>
+__global__ void __launch_bounds__(128) fm_candidate_simt_kernel(int32_t n_r, int32_t n_c, int32_t d, int32_t k,
+                                                                const T* __restrict__ XC, const T* __restrict__ P,
+                                                                const int32_t* __restrict__ row2req,
+                                                                const float* __restrict__ TT, T* __restrict__ FC) {
+  extern __shared__ float sm[];
+  const int32_t ds = d + 1;
+  float* xc = sm;                     // [n_c, d + 1]
+  float* ht = xc + (size_t)n_c * ds;  // [k, d + 1]
+  float* pc = ht + (size_t)k * ds;    // [n_c, k]
+  const int64_t i = blockIdx.x;
+  const int32_t r = row2req[i];
+  for (int e = threadIdx.x; e < n_c * d; e += blockDim.x) xc[(e / d) * ds + e % d] = ld_f(XC, i * n_c * d + e);
+  for (int e = threadIdx.x; e < n_c * k; e += blockDim.x) pc[e] = ld_f(P, (int64_t)n_r * k + e);
+  __syncthreads();
+  for (int idx = threadIdx.x; idx < k * d; idx += blockDim.x) {
+    const int c = idx / d, e = idx % d;
+    float acc = TT[((int64_t)r * k + c) * d + e];
+    for (int a = 0; a < n_c; ++a) acc = fmaf(pc[a * k + c], xc[a * ds + e], acc);
+    ht[c * ds + e] = acc;
+  }
+  __syncthreads();
+  for (int idx = threadIdx.x; idx < n_c * k; idx += blockDim.x) {
+    const int a = idx / k, c = idx % k;
+    float acc = 0.f;
+    for (int e = 0; e < d; ++e) acc = fmaf(xc[a * ds + e], ht[c * ds + e], acc);
+    st_f(FC, (i * n_c + a) * k + c, acc);
+  }
+}
+
+// ---------------------------------------------------------------------------------------------
+// Candidate side, bf16 streaming kernel: n_c = 16, k in {8, 16}, d a multiple of 64 up to 256.
+// ---------------------------------------------------------------------------------------------
+constexpr int kNc = 16;            // rows per candidate
+constexpr int kTileCands = 8;      // candidates per tile = compute warps per CTA
+constexpr int kTileRows = kNc * kTileCands;  // 128
+constexpr int kFmThreads = (kTileCands + 1) * 32;
+constexpr int kSlabBytes = kTileRows * 128;  // 64 columns of the tile, 128-byte swizzled rows
+constexpr uint32_t kStatusFm = 0x600;
+
+__device__ __forceinline__ void ldmatrix_x4(uint32_t addr, uint32_t (&r)[4]) {
+  asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0, %1, %2, %3}, [%4];"
+               : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3])
+               : "r"(addr));
+}
+__device__ __forceinline__ void ldmatrix_x4_trans(uint32_t addr, uint32_t (&r)[4]) {
+  asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0, %1, %2, %3}, [%4];"
+               : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3])
+               : "r"(addr));
+}
+__device__ __forceinline__ void mma_bf16(float (&c)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1) {
+  asm volatile(
+      "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0, %1, %2, %3}, {%4, %5, %6, %7}, {%8, %9}, "
+      "{%0, %1, %2, %3};"
+      : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
+      : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
+}
+__device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
+  const __nv_bfloat162 h = __floats2bfloat162_rn(lo, hi);
+  return *reinterpret_cast<const uint32_t*>(&h);
+}
+
+struct FmParams {
+  int64_t N;
+  int32_t n_r, k, num_tiles;
+  const __nv_bfloat16* P;        // [n_r + 16, k]
+  const int32_t* row2req;        // [N]
+  const float* TT;               // [R, k, d]
+  __nv_bfloat16* FC;             // [N, 16, k]
+  uint32_t* status;
+};
+
+template <int D, int STAGES>
+__global__ void __launch_bounds__(kFmThreads, 1)
+fm_candidate_mma_kernel(const __grid_constant__ CUtensorMap map_xc, const FmParams p) {
+  constexpr int kSlabs = D / 64;
+  constexpr int kStageBytes = kSlabs * kSlabBytes;
+  constexpr int kPairs = D / 16;  // pairs of 8-column groups = k-steps of step 2
+  extern __shared__ __align__(1024) uint8_t smem[];
+  uint64_t* full = reinterpret_cast<uint64_t*>(smem + STAGES * kStageBytes);
+  uint64_t* empty = full + STAGES;
+  AbortFlag* abort_flag = reinterpret_cast<AbortFlag*>(empty + STAGES);
+  const int warp = threadIdx.x / 32, lane = threadIdx.x % 32;
+  if ((smem_u32(smem) & 1023u) != 0) {  // the swizzled tiles assume a 1024-byte aligned base
+    if (threadIdx.x == 0) atomicCAS(p.status, 0u, kStatusFm | 15);
+    return;
+  }
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < STAGES; ++s) {
+      mbar_init(&full[s], 1);
+      mbar_init(&empty[s], kTileCands);
+    }
+    abort_flag->v = 0;
+    fence_mbar_init();
+  }
+  __syncthreads();
+
+  if (warp == kTileCands) {
+    // ------------------------------ TMA producer ------------------------------------------
+    if (lane == 0) {
+      prefetch_tensormap(&map_xc);
+      uint32_t it = 0;
+      for (int32_t t = blockIdx.x; t < p.num_tiles; t += gridDim.x, ++it) {
+        const int s = it % STAGES;
+        if (!mbar_wait(&empty[s], ((it / STAGES) & 1) ^ 1, abort_flag, p.status, kStatusFm | 1)) break;
+        mbar_expect_tx(&full[s], kStageBytes);
+#pragma unroll
+        for (int sl = 0; sl < kSlabs; ++sl)
+          tma_load_2d(smem + s * kStageBytes + sl * kSlabBytes, &map_xc, &full[s], sl * 64, t * kTileRows);
+      }
+      // loads in flight land in this CTA's shared memory: wait for them before the CTA may exit
+      for (int s = 0; s < STAGES; ++s) {
+        const uint32_t n_issued = it / STAGES + (((int)(it % STAGES) > s) ? 1 : 0);
+        if (n_issued == 0) continue;
+        const uint64_t t0 = globaltimer_ns();
+        while (!mbar_try_wait(&full[s], (n_issued - 1) & 1) && globaltimer_ns() - t0 < kWaitLimitNs) {}
+      }
+    }
+  } else {
+    // ------------------------------ one candidate per warp ---------------------------------
+    const int g = lane / 4, tq = lane % 4;  // fragment row group and column pair
+    // P_C^T as the M x K operand of step 1: A[m = projection column][kk = candidate row]
+    uint32_t pa[4];
+    {
+      const __nv_bfloat16* pc = p.P + (int64_t)p.n_r * p.k;
+      auto at = [&](int row, int col) -> float {  // P_C[row][col], zero beyond k columns
+        return col < p.k ? __bfloat162float(pc[row * p.k + col]) : 0.f;
+      };
+      pa[0] = pack_bf16(at(2 * tq, g), at(2 * tq + 1, g));
+      pa[1] = pack_bf16(at(2 * tq, g + 8), at(2 * tq + 1, g + 8));
+      pa[2] = pack_bf16(at(2 * tq + 8, g), at(2 * tq + 9, g));
+      pa[3] = pack_bf16(at(2 * tq + 8, g + 8), at(2 * tq + 9, g + 8));
+    }
+    // this lane's address pattern inside a candidate's 16 rows: row, and which of the two
+    // 8-column groups of a pair
+    const int lrow = (lane % 8) + ((lane / 8) % 2) * 8;
+    const int lsel = lane / 16;
+    float tfrag[kPairs][2][4];  // T^T of the cached request in step-1 accumulator layout
+    int32_t cached_req = -1;
+    uint32_t it = 0;
+    for (int32_t t = blockIdx.x; t < p.num_tiles; t += gridDim.x, ++it) {
+      const int s = it % STAGES;
+      if (!mbar_wait(&full[s], (it / STAGES) & 1, abort_flag, p.status, kStatusFm | 2)) break;
+      const int64_t cand = (int64_t)t * kTileCands + warp;
+      if (cand < p.N) {
+        const int32_t r = p.row2req[cand];
+        if (r != cached_req) {
+          cached_req = r;
+          const float* tt = p.TT + (int64_t)r * p.k * D;
+#pragma unroll
+          for (int cp = 0; cp < kPairs; ++cp)
+#pragma unroll
+            for (int h = 0; h < 2; ++h) {
+              const int col = (2 * cp + h) * 8 + 2 * tq;
+              const float2 lo = g < p.k ? *reinterpret_cast<const float2*>(tt + g * D + col) : make_float2(0.f, 0.f);
+              const float2 hi = g + 8 < p.k ? *reinterpret_cast<const float2*>(tt + (g + 8) * D + col) : make_float2(0.f, 0.f);
+              tfrag[cp][h][0] = lo.x;
+              tfrag[cp][h][1] = lo.y;
+              tfrag[cp][h][2] = hi.x;
+              tfrag[cp][h][3] = hi.y;
+            }
+        }
+        const uint32_t tile = smem_u32(smem + s * kStageBytes);
+        const int trow = warp * kNc + lrow;
+        // step 1: H^T (16 x D) = T^T + P_C^T X^C, rounded to bf16 as the K x N operand of step 2
+        uint32_t hb[kPairs][2][2];  // [k-step][projection columns 0-7 | 8-15][b0, b1]
+#pragma unroll
+        for (int cp = 0; cp < kPairs; ++cp) {
+          const int chunk = 2 * cp + lsel;  // 16-byte chunk along d
+          uint32_t xb[4];
+          ldmatrix_x4_trans(tile + (chunk / 8) * kSlabBytes + trow * 128 + (((chunk % 8) ^ (trow & 7)) << 4), xb);
+          float acc0[4], acc1[4];
+#pragma unroll
+          for (int e = 0; e < 4; ++e) {
+            acc0[e] = tfrag[cp][0][e];
+            acc1[e] = tfrag[cp][1][e];
+          }
+          mma_bf16(acc0, pa, xb[0], xb[1]);
+          mma_bf16(acc1, pa, xb[2], xb[3]);
+          hb[cp][0][0] = pack_bf16(acc0[0], acc0[1]);
+          hb[cp][0][1] = pack_bf16(acc1[0], acc1[1]);
+          hb[cp][1][0] = pack_bf16(acc0[2], acc0[3]);
+          hb[cp][1][1] = pack_bf16(acc1[2], acc1[3]);
+        }
+        // step 2: FC (16 x 16) = X^C H
+        float out0[4] = {0.f, 0.f, 0.f, 0.f}, out1[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+        for (int cp = 0; cp < kPairs; ++cp) {
+          const int chunk = 2 * cp + lsel;
+          uint32_t xa[4];
+          ldmatrix_x4(tile + (chunk / 8) * kSlabBytes + trow * 128 + (((chunk % 8) ^ (trow & 7)) << 4), xa);
+          mma_bf16(out0, xa, hb[cp][0][0], hb[cp][0][1]);
+          mma_bf16(out1, xa, hb[cp][1][0], hb[cp][1][1]);
+        }
+        __nv_bfloat16* fc = p.FC + cand * kNc * p.k;
+        *reinterpret_cast<uint32_t*>(fc + g * p.k + 2 * tq) = pack_bf16(out0[0], out0[1]);
+        *reinterpret_cast<uint32_t*>(fc + (g + 8) * p.k + 2 * tq) = pack_bf16(out0[2], out0[3]);
+        if (p.k > 8) {
+          *reinterpret_cast<uint32_t*>(fc + g * p.k + 8 + 2 * tq) = pack_bf16(out1[0], out1[1]);
+          *reinterpret_cast<uint32_t*>(fc + (g + 8) * p.k + 8 + 2 * tq) = pack_bf16(out1[2], out1[3]);
+        }
+      }
+      __syncwarp();
+      if (lane == 0) mbar_arrive(&empty[s]);
+    }
+  }
+}
+
+int sm_count_fm() {
+  static int n = 0;
+  if (n == 0) {
+    int dev = 0;
+    cudaGetDevice(&dev);
+    cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev);
+  }
+  return n;
+}
+
+template <int D>
+rocs_status_t launch_fm_mma(const rocs_plan* plan, int32_t n_r, int32_t k, const void* XC, const void* P,
+                            const float* TT, void* FC, cudaStream_t stream) {
+  constexpr int kStages = D <= 64 ? 8 : D <= 128 ? 6 : 3;
+  constexpr int kSmem = kStages * (D / 64) * kSlabBytes + 512;
+  CUtensorMap map_xc;
+  if (!make_tensor_map_2d(&map_xc, XC, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, (uint64_t)plan->N * kNc, D, D, kTileRows, 64,
+                          true))
+    return ROCS_ERR_CUDA;
+  uint32_t* status = device_status_word();
+  if (!status) return ROCS_ERR_CUDA;
+  FmParams p{};
+  p.N = plan->N;
+  p.n_r = n_r;
+  p.k = k;
+  p.num_tiles = (int32_t)((plan->N + kTileCands - 1) / kTileCands);
+  p.P = (const __nv_bfloat16*)P;
+  p.row2req = plan->row2req;
+  p.TT = TT;
+  p.FC = (__nv_bfloat16*)FC;
+  p.status = status;
+  auto kern = fm_candidate_mma_kernel<D, kStages>;
+  ROCS_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmem));
+  const int grid = std::min(p.num_tiles, sm_count_fm());
+  kern<<<grid, kFmThreads, kSmem, stream>>>(map_xc, p);
+  ROCS_CUDA_TRY(cudaGetLastError());
+  return ROCS_OK;
+}
+
+template <typename T>
+rocs_status_t launch_fm(const rocs_plan* plan, int32_t n_r, int32_t n_c, int32_t d, int32_t k, const void* XR,
+                        const void* XC, const void* P, void* FR, void* FC, float* TT, bool fast_candidates,
+                        cudaStream_t stream) {
+  constexpr size_t kMaxSmem = 200 * 1024;
+  const size_t smem_r = ((size_t)(n_r + k) * (d + 1) + (size_t)n_r * k) * sizeof(float);
+  const size_t smem_c = ((size_t)(n_c + k) * (d + 1) + (size_t)n_c * k) * sizeof(float);
+  if (smem_r > kMaxSmem || smem_c > kMaxSmem) return ROCS_ERR_UNSUPPORTED;
+  if (plan->R > 0) {
+    ROCS_CUDA_TRY(cudaFuncSetAttribute(fm_request_kernel<T>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kMaxSmem));
+    fm_request_kernel<T><<<plan->R, 256, smem_r, stream>>>(n_r, d, k, (const T*)XR, (const T*)P, TT, (T*)FR);
+    ROCS_CUDA_TRY(cudaGetLastError());
+  }
+  if (plan->N == 0 || !FC) return ROCS_OK;
+  if (fast_candidates) {
+    switch (d) {
+      case 64: return launch_fm_mma<64>(plan, n_r, k, XC, P, TT, FC, stream);
+      case 128: return launch_fm_mma<128>(plan, n_r, k, XC, P, TT, FC, stream);
+      case 192: return launch_fm_mma<192>(plan, n_r, k, XC, P, TT, FC, stream);
+      case 256: return launch_fm_mma<256>(plan, n_r, k, XC, P, TT, FC, stream);
+      default: break;
+    }
+  }
+  ROCS_CUDA_TRY(cudaFuncSetAttribute(fm_candidate_simt_kernel<T>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kMaxSmem));
+  fm_candidate_simt_kernel<T><<<(unsigned)plan->N, 128, smem_c, stream>>>(n_r, n_c, d, k, (const T*)XC, (const T*)P,
+                                                                         plan->row2req, TT, (T*)FC);
+  ROCS_CUDA_TRY(cudaGetLastError());
+  return ROCS_OK;
+}
+
+}  // namespace
+
+bool fm_projection_fast_supported(int32_t n_c, int32_t d, int32_t k) {
+  return n_c == kNc && (k == 8 || k == 16) && d % 64 == 0 && d >= 64 && d <= 256;
+}
+
+rocs_status_t fm_projection(rocs_dtype_t dt, const rocs_plan* plan, int32_t n_r, int32_t n_c, int32_t d, int32_t k,
+                            const void* XR, const void* XC, const void* P, void* FR, void* FC, float* tt_workspace,
+                            bool allow_fast, cudaStream_t stream) {
+  if (dt == ROCS_F32)
+    return launch_fm<float>(plan, n_r, n_c, d, k, XR, XC, P, FR, FC, tt_workspace, false, stream);
+  return launch_fm<__nv_bfloat16>(plan, n_r, n_c, d, k, XR, XC, P, FR, FC, tt_workspace,
+                                  allow_fast && fm_projection_fast_supported(n_c, d, k), stream);
+}
+
+}  // namespace rocs

@@ -91,6 +91,14 @@ rocs_status_t simt_glm(rocs_dtype_t dt, const rocs_plan* plan, int32_t n_r, int3
                        void* YR, void* YC, void* OR_, void* OC, float* zr_workspace,
                        cudaStream_t stream);
 
+// ---- projected factorization machine: fm_projection.cu ----------------------------------
+// F = G P on the request-once form; tt_workspace [R, k, d] fp32 receives P_R^T X^R per request.
+// allow_fast: use the bf16 streaming kernel for the candidate side where the shape allows it.
+bool fm_projection_fast_supported(int32_t n_c, int32_t d, int32_t k);
+rocs_status_t fm_projection(rocs_dtype_t dt, const rocs_plan* plan, int32_t n_r, int32_t n_c, int32_t d, int32_t k,
+                            const void* XR, const void* XC, const void* P, void* FR, void* FC, float* tt_workspace,
+                            bool allow_fast, cudaStream_t stream);
+
 // ---- tcgen05 tensor-core kernels (bf16): umma_*.cu -------------------------------------
 bool umma_linear_supported(int64_t M, int32_t d_in, int32_t d_out, int64_t ld_x, int64_t ld_w,
                            int64_t ld_y, bool out_f32);
