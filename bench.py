@@ -415,6 +415,8 @@ def bench_other_ops(torch, rocs, peaks, dev, time_call, which=("dca", "glm")):
         out.append(bench_dca(torch, rocs, peaks, dev, time_call))
     if "glm" in which:
         out.append(bench_glm(torch, rocs, peaks, dev, time_call))
+    if "fm" in which:
+        out.append(bench_fm(torch, rocs, peaks, dev, time_call))
     if "cfg5" in which:
         out.extend(bench_cfg5(torch, rocs, peaks, dev, time_call))
     return out
@@ -508,6 +510,37 @@ def bench_glm(torch, rocs, peaks, dev, time_call):
             "note": "input (537 MB) is larger than L2; same buffers every iteration"}
 
 
+def materialised_fm(torch, XR, XC, P, counts_dev, n_r):
+    """X = [X^R[m_i]; X^C[i]] per candidate, G = X X^T, block mask, F = G P (candidate rows)."""
+    X = torch.cat([XR.repeat_interleave(counts_dev, dim=0), XC], dim=1)
+    G = torch.bmm(X[:, n_r:], X.transpose(1, 2))
+    return torch.matmul(G, P)
+
+
+def bench_fm(torch, rocs, peaks, dev, time_call):
+    # configuration 4 shapes: projected factorization machine, k = 16
+    cfg = wl.CONFIGS[4]
+    k = 16
+    co = wl.cand_offsets(cfg)
+    N = int(co[-1])
+    d = wl.glm_inputs(cfg, co)
+    plan4 = rocs.plan_create(dev(co), co)
+    XR, XC, P = dev(d["XR"]), dev(d["XC"]), dev(wl.fm_projection_weight(cfg, k))
+    outs = {"FC": torch.empty((N, cfg.n_c, k), dtype=torch.bfloat16, device="cuda"),
+            "FR": torch.empty((cfg.R, cfg.n_r, k), dtype=torch.bfloat16, device="cuda")}
+    ws = torch.empty(rocs.glm_fm_projection_workspace(plan4, cfg.d_emb, k), dtype=torch.uint8, device="cuda")
+    t = time_call(lambda i: rocs.glm_fm_projection(plan4, XR, XC, P, workspace=ws, outs=outs), reps=10)
+    nbytes = XC.numel() * 2 + outs["FC"].numel() * 2 + XR.numel() * 2
+    flops = N * 4.0 * cfg.n_c * cfg.d_emb * k
+    counts_dev = dev(np.diff(co).astype(np.int64))
+    t_mat = time_call(lambda i: materialised_fm(torch, XR, XC, P, counts_dev, cfg.n_r), reps=3)
+    return {"layer": "cfg4 shapes glm_fm_projection 32+16 x128 -> k=16", "N": N, "us": t * 1e6,
+            "materialised_broadcast_gpu_us": t_mat * 1e6, "speedup_vs_materialised": t_mat / t,
+            "cand_per_s": N / t, "gbs": nbytes / t / 1e9, "frac_hbm": nbytes / t / 1e9 / peaks["hbm_gbs"],
+            "tflops": flops / t / 1e12,
+            "note": "input (537 MB) is larger than L2; same buffers every iteration"}
+
+
 def bench_cfg5(torch, rocs, peaks, dev, time_call):
     """Configuration 5 (skewed, Zipf candidate counts): the three calls timed independently."""
     cfg = wl.CONFIGS[5]
@@ -561,7 +594,7 @@ def main():
     ap.add_argument("--warmup", type=int, default=10)
     ap.add_argument("--impl", default="rocs", choices=["rocs", "reference"])
     ap.add_argument("--skip-extra", action="store_true", help="skip the attention / interaction side measurements")
-    ap.add_argument("--extra", default="dca,glm", help="side measurements to run: dca, glm, cfg5")
+    ap.add_argument("--extra", default="dca,glm", help="side measurements to run: dca, glm, fm, cfg5")
     ap.add_argument("--skip-cpu", action="store_true", help="skip the cpu_baseline leg")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "rocs" else args.warmup

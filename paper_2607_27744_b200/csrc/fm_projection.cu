@@ -164,13 +164,18 @@ fm_candidate_mma_kernel(const __grid_constant__ CUtensorMap map_xc, const FmPara
     fence_mbar_init();
   }
   __syncthreads();
+  // a contiguous run of tiles per CTA: consecutive candidates mostly share their request, so the
+  // request's T block is reloaded only where a segment ends
+  const int32_t tiles_per_cta = (p.num_tiles + (int32_t)gridDim.x - 1) / (int32_t)gridDim.x;
+  const int32_t tile_begin = min((int32_t)blockIdx.x * tiles_per_cta, p.num_tiles);
+  const int32_t tile_end = min(tile_begin + tiles_per_cta, p.num_tiles);
 
   if (warp == kTileCands) {
     // ------------------------------ TMA producer ------------------------------------------
     if (lane == 0) {
       prefetch_tensormap(&map_xc);
       uint32_t it = 0;
-      for (int32_t t = blockIdx.x; t < p.num_tiles; t += gridDim.x, ++it) {
+      for (int32_t t = tile_begin; t < tile_end; ++t, ++it) {
         const int s = it % STAGES;
         if (!mbar_wait(&empty[s], ((it / STAGES) & 1) ^ 1, abort_flag, p.status, kStatusFm | 1)) break;
         mbar_expect_tx(&full[s], kStageBytes);
@@ -208,7 +213,7 @@ fm_candidate_mma_kernel(const __grid_constant__ CUtensorMap map_xc, const FmPara
     float tfrag[kPairs][2][4];  // T^T of the cached request in step-1 accumulator layout
     int32_t cached_req = -1;
     uint32_t it = 0;
-    for (int32_t t = blockIdx.x; t < p.num_tiles; t += gridDim.x, ++it) {
+    for (int32_t t = tile_begin; t < tile_end; ++t, ++it) {
       const int s = it % STAGES;
       if (!mbar_wait(&full[s], (it / STAGES) & 1, abort_flag, p.status, kStatusFm | 2)) break;
       const int64_t cand = (int64_t)t * kTileCands + warp;
