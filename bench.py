@@ -415,6 +415,8 @@ def bench_other_ops(torch, rocs, peaks, dev, time_call, which=("dca", "glm")):
         out.append(bench_dca(torch, rocs, peaks, dev, time_call))
     if "glm" in which:
         out.append(bench_glm(torch, rocs, peaks, dev, time_call))
+    if "nq" in which:
+        out.append(bench_dca_nq(torch, rocs, peaks, dev, time_call))
     if "fm" in which:
         out.append(bench_fm(torch, rocs, peaks, dev, time_call))
     if "cfg5" in which:
@@ -483,6 +485,26 @@ def bench_dca(torch, rocs, peaks, dev, time_call):
             "bound": "tensor (nominal); the exponential unit (16 ex2/clk/SM) is the tighter ceiling at dh = 64",
             "frac_of_exp_unit_peak_at_max_clock": pairs * cfg.H / t / (148 * 16 * 1.965e9),
             "frac_tensor_sustained": flops / t / 1e12 / peaks["tflops_sustained"]}
+
+
+def bench_dca_nq(torch, rocs, peaks, dev, time_call, n_q=32):
+    """Multi-token candidate queries (Section 4.3.2): configuration 3 with n_q query tokens per
+    candidate and 1/n_q as many candidates per request, so the query rows and flops stay put."""
+    base = wl.CONFIGS[3]
+    cfg = base.with_(n_q=n_q)
+    counts = np.maximum(1, np.diff(wl.cand_offsets(base)) // n_q)
+    co, so = wl.offsets_from_counts(counts.tolist()), wl.seq_offsets(base)
+    N = int(co[-1])
+    d = wl.dca_inputs(cfg, co, so)
+    plan = rocs.plan_create(dev(co), co)
+    Q, K, V, sod = dev(d["Q"]), dev(d["K"]), dev(d["V"]), dev(so)
+    O = torch.empty_like(Q)
+    t = time_call(lambda i: rocs.dca_attention(plan, Q, K, V, sod, out=O), reps=5)
+    pairs = float(np.sum(np.diff(co).astype(np.float64) * np.diff(so))) * n_q
+    flops = 4.0 * pairs * cfg.H * cfg.dh
+    return {"layer": f"cfg3 dca_attention with n_q={n_q} query tokens per candidate (R=64, L=2048, 8x64)", "N": N,
+            "us": t * 1e6, "cand_per_s": N / t, "query_rows_per_s": N * n_q / t, "tflops": flops / t / 1e12,
+            "frac_tensor": flops / t / 1e12 / peaks["tflops_burst"], "exps_per_s": pairs * cfg.H / t}
 
 
 def bench_glm(torch, rocs, peaks, dev, time_call):
@@ -594,7 +616,7 @@ def main():
     ap.add_argument("--warmup", type=int, default=10)
     ap.add_argument("--impl", default="rocs", choices=["rocs", "reference"])
     ap.add_argument("--skip-extra", action="store_true", help="skip the attention / interaction side measurements")
-    ap.add_argument("--extra", default="dca,glm", help="side measurements to run: dca, glm, fm, cfg5")
+    ap.add_argument("--extra", default="dca,glm", help="side measurements to run: dca, nq, glm, fm, cfg5")
     ap.add_argument("--skip-cpu", action="store_true", help="skip the cpu_baseline leg")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "rocs" else args.warmup
