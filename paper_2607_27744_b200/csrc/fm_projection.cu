@@ -45,6 +45,9 @@ __global__ void __launch_bounds__(256) fm_request_kernel(int32_t n_r, int32_t d,
   float* tt = xr + (size_t)n_r * ds;  // [k, d + 1]
   float* pr = tt + (size_t)k * ds;    // [n_r, k]
   const int32_t r = blockIdx.x;
+  // the candidate kernel may start now: it streams X^C on its own and waits for this grid only
+  // before it reads TT
+  ptx::griddep_launch_dependents();
   for (int e = threadIdx.x; e < n_r * d; e += blockDim.x) xr[(e / d) * ds + e % d] = ld_f(XR, (int64_t)r * n_r * d + e);
   for (int e = threadIdx.x; e < n_r * k; e += blockDim.x) pr[e] = ld_f(P, e);
   __syncthreads();
@@ -220,6 +223,7 @@ fm_candidate_mma_kernel(const __grid_constant__ CUtensorMap map_xc, const FmPara
       if (cand < p.N) {
         const int32_t r = p.row2req[cand];
         if (r != cached_req) {
+          if (cached_req < 0) griddep_wait();  // TT comes from the request kernel launched just before
           cached_req = r;
           const float* tt = p.TT + (int64_t)r * p.k * D;
 #pragma unroll
@@ -314,9 +318,19 @@ rocs_status_t launch_fm_mma(const rocs_plan* plan, int32_t n_r, int32_t k, const
   p.status = status;
   auto kern = fm_candidate_mma_kernel<D, kStages>;
   ROCS_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmem));
-  const int grid = std::min(p.num_tiles, sm_count_fm());
-  kern<<<grid, kFmThreads, kSmem, stream>>>(map_xc, p);
-  ROCS_CUDA_TRY(cudaGetLastError());
+  // Launched so that it may overlap the request kernel in front of it on the stream (that kernel
+  // releases its dependents at once); nothing else this kernel reads is written by that launch.
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3((unsigned)std::min(p.num_tiles, sm_count_fm()));
+  cfg.blockDim = dim3(kFmThreads);
+  cfg.dynamicSmemBytes = kSmem;
+  cfg.stream = stream;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  ROCS_CUDA_TRY(cudaLaunchKernelEx(&cfg, kern, map_xc, p));
   return ROCS_OK;
 }
 
