@@ -6,7 +6,11 @@
 // its own TMEM.  Parking only half a slice per SM (64 KB at d_in = 256) leaves shared memory for a
 // deep X ring AND a swizzled staging area, so the output leaves through TMA stores: the epilogue
 // spends shared-memory wavefronts on 16-byte row pieces instead of one global-memory wavefront per
-// 32-byte piece, which is what bounds the single-CTA variant.
+// 32-byte piece, which is what bounds the single-CTA variant (measured here as well: the same
+// epilogue with 32-byte register stores runs in 107 us instead of 84 on configuration 2).  The X ring
+// is what the time is most sensitive to (2 / 3 / 4 / 5 / 7 stages: 127 / 107 / 93 / 86 / 84 us), so
+// each epilogue warp stages through ONE 4 KB box, used for both of its 64-column chunks, and the
+// shared memory saved goes to the ring.
 //
 //   pair P: column slice P % n_slices, row group P / n_slices; super-tiles (256 rows) g, g + G, ...
 //   warp 0 (both CTAs)  TMA producer: its half of W once; per tile its X tile (k_blocks x 16 KB,
@@ -34,7 +38,7 @@ constexpr int kAStageBytes = BM * BK * 2;        // 16 KB
 constexpr int kWBlockBytes = (BN / 2) * BK * 2;  // this CTA's half of a 64-wide K block: 16 KB
 constexpr int kZBufBytes = 4 * BN * 4;           // four slabs x 256 fp32
 constexpr int kZBufs = 4;                        // request-row buffers: the producer may run this many tiles ahead
-constexpr int kStagingBytes = kEpiWarps * 8192;  // per warp: two 32-row x 128-byte boxes
+constexpr int kStagingBytes = kEpiWarps * 4096;  // per warp: one 32-row x 128-byte box, reused by both column chunks
 constexpr uint32_t kStatusWs2 = 0x500;
 
 struct Ws2Params {
@@ -202,7 +206,7 @@ linear_ws2_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_consta
     // ------------------------------ epilogue (both CTAs) ------------------------------------
     const int q = warp % 4;             // TMEM lane quadrant = 32-row slab of this CTA's 128 rows
     const int half = (warp - 2) / 4;    // which 128 of the slice's 256 columns
-    uint8_t* my_stage = staging + (warp - 2) * 8192;
+    uint8_t* my_stage = staging + (warp - 2) * 4096;
     const uint32_t tmem_empty_leader[2] = {map_to_cta(smem_u32(&tmem_empty[0]), 0),
                                            map_to_cta(smem_u32(&tmem_empty[1]), 0)};
     uint32_t lt = 0;
@@ -272,7 +276,11 @@ linear_ws2_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_consta
 #pragma unroll
           for (int i = 0; i < 64; ++i) f[i] = fmaxf(f[i], 0.f);
         }
-        uint8_t* row_ptr = my_stage + c * 4096 + lane * 128;
+        if (c == 1) {  // the store of the first chunk has finished reading the box
+          if (lane == 0) tma_store_wait_read<0>();
+          __syncwarp();
+        }
+        uint8_t* row_ptr = my_stage + lane * 128;
 #pragma unroll
         for (int j = 0; j < 8; ++j) {  // eight 16-byte pieces per 128-byte row, XOR-swizzled by row
           uint4 w;
@@ -286,17 +294,15 @@ linear_ws2_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_consta
           w.w = *reinterpret_cast<uint32_t*>(&h3);
           *reinterpret_cast<uint4*>(row_ptr + ((j ^ (lane & 7)) << 4)) = w;
         }
-      }
-      fence_proxy_async_smem();
-      __syncwarp();
-      if (lane == 0) {
-#pragma unroll
-        for (int c = 0; c < 2; ++c)
+        fence_proxy_async_smem();
+        __syncwarp();
+        if (lane == 0) {
           if (n0 + half * 128 + c * 64 < p.d_out && (int64_t)m0 + q * 32 < p.M)
-            tma_store_2d(&map_y, my_stage + c * 4096, n0 + half * 128 + c * 64, m0 + q * 32);
-        tma_store_commit();
-        if (has_add) mbar_arrive(&z_empty[lt % kZBufs]);
+            tma_store_2d(&map_y, my_stage, n0 + half * 128 + c * 64, m0 + q * 32);
+          tma_store_commit();
+        }
       }
+      if (lane == 0 && has_add) mbar_arrive(&z_empty[lt % kZBufs]);
     }
     if (lane == 0) tma_store_wait_all<0>();
   }
