@@ -476,3 +476,41 @@ int rocs_ref_glm_fm_projection_decomposed(int dtype, int32_t R, int64_t N, const
   free(H);
   return 0;
 }
+
+/* ------------------------------------------------------------------------- *
+ * Group-local normalisation (Eq. 7): y^(i) = Norm_i(x^(i)), one group's tensor
+ * at a time, so no statistic ever spans two groups.  X [M, d]; every row is
+ * normalised over its d coordinates.
+ *   kind 0  LayerNorm:  y = (x - mean) / sqrt(var + eps) * gamma + beta   (biased variance)
+ *   kind 1  RMSNorm:    y = x / sqrt(mean(x^2) + eps) * gamma             (beta ignored)
+ * gamma / beta may be NULL (1 / 0).  Y_out [M, d] fp64.
+ * ------------------------------------------------------------------------- */
+int rocs_ref_group_norm(int dtype, int64_t M, int32_t d, const void *X, const void *gamma, const void *beta,
+                        double eps, int kind, double *Y_out) {
+  if (kind != 0 && kind != 1) return -1;
+#pragma omp parallel for schedule(static)
+  for (int64_t i = 0; i < M; ++i) {
+    double mean = 0.0, sq = 0.0;
+    for (int32_t e = 0; e < d; ++e) mean += load_as_f64(X, dtype, i * d + e);
+    mean /= d;
+    if (kind == 0) {
+      for (int32_t e = 0; e < d; ++e) {
+        const double c = load_as_f64(X, dtype, i * d + e) - mean;
+        sq += c * c;
+      }
+    } else {
+      for (int32_t e = 0; e < d; ++e) {
+        const double v = load_as_f64(X, dtype, i * d + e);
+        sq += v * v;
+      }
+    }
+    const double inv = 1.0 / sqrt(sq / d + eps);
+    for (int32_t e = 0; e < d; ++e) {
+      const double g = gamma ? load_as_f64(gamma, dtype, e) : 1.0;
+      const double b = (beta && kind == 0) ? load_as_f64(beta, dtype, e) : 0.0;
+      const double v = load_as_f64(X, dtype, i * d + e);
+      Y_out[i * d + e] = (kind == 0 ? (v - mean) : v) * inv * g + b;
+    }
+  }
+  return 0;
+}

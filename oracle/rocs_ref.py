@@ -241,3 +241,18 @@ def glm_fm_projection_decomposed(cand_offsets, XR, XC, P):
         dt, R, ctypes.c_int64(N), _ptr(co), n_r, n_c, d, k, _ptr(XR), _ptr(XC), _ptr(P), _ptr(FR), _ptr(FC))
     assert rc == 0
     return FR, FC
+
+
+LAYER_NORM, RMS_NORM = 0, 1
+
+
+def group_norm(X, gamma=None, beta=None, eps=1e-5, kind=LAYER_NORM):
+    """Eq. 7 on one group's tensor X [M, d]: LayerNorm (biased variance) or RMSNorm over each row."""
+    X, gamma, beta = _c(X), _c(gamma), _c(beta)
+    M, d = X.shape
+    dt = _same_dtype(X, gamma, beta)
+    Y = np.empty((M, d), np.float64)
+    rc = _load().rocs_ref_group_norm(dt, ctypes.c_int64(M), d, _ptr(X), _ptr(gamma), _ptr(beta),
+                                     ctypes.c_double(eps), kind, _ptr(Y))
+    assert rc == 0
+    return Y
