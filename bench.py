@@ -419,6 +419,8 @@ def bench_other_ops(torch, rocs, peaks, dev, time_call, which=("dca", "glm")):
         out.append(bench_dca_nq(torch, rocs, peaks, dev, time_call))
     if "fm" in which:
         out.append(bench_fm(torch, rocs, peaks, dev, time_call))
+    if "norm" in which:
+        out.append(bench_norm(torch, rocs, peaks, dev, time_call))
     if "cfg5" in which:
         out.extend(bench_cfg5(torch, rocs, peaks, dev, time_call))
     return out
@@ -563,6 +565,22 @@ def bench_fm(torch, rocs, peaks, dev, time_call):
             "note": "input (537 MB) is larger than L2; same buffers every iteration"}
 
 
+def bench_norm(torch, rocs, peaks, dev, time_call):
+    # group-local RMSNorm (Eq. 7) of the candidate-side activations of configuration 2: 131072 x 1024
+    cfg = wl.CONFIGS[2]
+    N = cfg.R * cfg.count_const
+    g = torch.Generator(device="cuda").manual_seed(7)
+    X = torch.randn(N, cfg.d_out, generator=g, device="cuda", dtype=torch.float32).to(torch.bfloat16)
+    gamma = torch.ones(cfg.d_out, dtype=torch.bfloat16, device="cuda")
+    Y = torch.empty_like(X)
+    t = time_call(lambda i: rocs.group_norm(X, gamma, None, 1e-6, rocs.NORM_RMS, out=Y), reps=20)
+    nbytes = 2 * X.numel() * 2
+    t_lib = time_call(lambda i: torch.nn.functional.rms_norm(X, (cfg.d_out,), gamma, eps=1e-6), reps=20)
+    return {"layer": "cfg2 activations group_norm (RMSNorm, 131072 x 1024)", "N": N, "us": t * 1e6, "cand_per_s": N / t,
+            "gbs": nbytes / t / 1e9, "frac_hbm": nbytes / t / 1e9 / peaks["hbm_gbs"], "torch_rms_norm_us": t_lib * 1e6,
+            "note": "input and output (537 MB) are larger than L2"}
+
+
 def bench_cfg5(torch, rocs, peaks, dev, time_call):
     """Configuration 5 (skewed, Zipf candidate counts): the three calls timed independently."""
     cfg = wl.CONFIGS[5]
@@ -616,7 +634,7 @@ def main():
     ap.add_argument("--warmup", type=int, default=10)
     ap.add_argument("--impl", default="rocs", choices=["rocs", "reference"])
     ap.add_argument("--skip-extra", action="store_true", help="skip the attention / interaction side measurements")
-    ap.add_argument("--extra", default="dca,glm", help="side measurements to run: dca, nq, glm, fm, cfg5")
+    ap.add_argument("--extra", default="dca,glm", help="side measurements to run: dca, nq, glm, fm, norm, cfg5")
     ap.add_argument("--skip-cpu", action="store_true", help="skip the cpu_baseline leg")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "rocs" else args.warmup

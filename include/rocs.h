@@ -228,6 +228,21 @@ rocs_status_t rocs_glm_fm_projection(const rocs_plan_t* plan, rocs_dtype_t dtype
                                      void* workspace, size_t workspace_bytes, void* stream);
 
 /*
+ * Group-local normalisation (Eq. 7): y = Norm(x) on ONE group's tensor, every row over its own d
+ * coordinates, so no statistic spans two groups (normalise the request rows and the candidate rows
+ * with separate calls; statistics over concatenated groups would break the invariant of Eq. 1).
+ *     ROCS_NORM_LAYER:  y = (x - mean) / sqrt(var + eps) * gamma + beta    (biased variance)
+ *     ROCS_NORM_RMS:    y = x / sqrt(mean(x^2) + eps) * gamma              (beta is ignored)
+ *   X [M, d] with row stride ld_x, Y [M, d] with row stride ld_y (elements; Y may alias X)
+ *   gamma, beta [d] in the storage type, either may be NULL (1 and 0);  eps >= 0
+ * Statistics are accumulated in fp32.  Errors: INVALID_ARG, ALIGNMENT, CUDA.
+ */
+typedef enum { ROCS_NORM_LAYER = 0, ROCS_NORM_RMS = 1 } rocs_norm_t;
+rocs_status_t rocs_group_norm(rocs_dtype_t dtype, rocs_norm_t kind, int64_t M, int32_t d, const void* X,
+                              int64_t ld_x, const void* gamma, const void* beta, float eps, void* Y,
+                              int64_t ld_y, void* stream);
+
+/*
  * Device-side status of the tensor-core kernels.  Their barrier waits are bounded; a wait
  * that expires records a code in a device word instead of spinning forever and the kernel
  * returns.  This call synchronises the device, reads the word, clears it and returns

@@ -24,12 +24,13 @@ OK = 0
 BF16, F32 = 0, 1
 ACT_NONE, ACT_RELU = 0, 1
 PATH_AUTO, PATH_GENERAL = 0, 1
+NORM_LAYER, NORM_RMS = 0, 1
 
 EXPORTS = [
     "rocs_status_string", "rocs_padded_ld", "rocs_set_path", "rocs_plan_create", "rocs_plan_destroy",
     "rocs_ikbo_linear_workspace", "rocs_ikbo_linear", "rocs_linear", "rocs_dca_attention_workspace",
     "rocs_dca_attention", "rocs_glm_interaction_workspace", "rocs_glm_interaction",
-    "rocs_glm_fm_projection_workspace", "rocs_glm_fm_projection",
+    "rocs_glm_fm_projection_workspace", "rocs_glm_fm_projection", "rocs_group_norm",
     "rocs_last_device_status", "rocs_ikbo_linear_static", "rocs_ikbo_linear_static_max_z_elems",
     "rocs_ikbo_linear_static_max_candidates",
 ]
@@ -73,6 +74,7 @@ def lib() -> ctypes.CDLL:
         L.rocs_glm_fm_projection_workspace.restype = sz
         L.rocs_glm_fm_projection_workspace.argtypes = [vp, i32, i32]
         L.rocs_glm_fm_projection.argtypes = [vp, ctypes.c_int, i32, i32, i32, i32, vp, vp, vp, vp, vp, vp, sz, vp]
+        L.rocs_group_norm.argtypes = [ctypes.c_int, ctypes.c_int, i64, i32, vp, i64, vp, vp, f32, vp, i64, vp]
         L.rocs_last_device_status.argtypes = [ctypes.POINTER(ctypes.c_uint32)]
         L.rocs_ikbo_linear_static_max_z_elems.restype = sz
         L.rocs_ikbo_linear_static_max_candidates.restype = sz
@@ -284,6 +286,19 @@ def glm_fm_projection(plan: Plan, XR: torch.Tensor, XC: torch.Tensor, P: torch.T
         _p(workspace), workspace.numel(), _stream())
     _check(code, "rocs_glm_fm_projection")
     return outs
+
+
+def group_norm(X: torch.Tensor, gamma: Optional[torch.Tensor] = None, beta: Optional[torch.Tensor] = None,
+               eps: float = 1e-5, kind: int = NORM_LAYER, out: Optional[torch.Tensor] = None) -> torch.Tensor:
+    """Group-local LayerNorm / RMSNorm (Eq. 7) of one group's tensor X [M, d], row by row."""
+    assert X.dim() == 2 and X.stride(1) == 1
+    M, d = X.shape
+    if out is None:
+        out = torch.empty((M, d), dtype=X.dtype, device=X.device)
+    code = lib().rocs_group_norm(_dtype_code(X), kind, M, d, _p(X), _rows_2d(X), _p(gamma), _p(beta), eps, _p(out),
+                                 _rows_2d(out), _stream())
+    _check(code, "rocs_group_norm")
+    return out
 
 
 def ikbo_linear_static(cand_offsets: torch.Tensor, XR: torch.Tensor, XC: torch.Tensor, W_CR: torch.Tensor,

@@ -370,6 +370,20 @@ rocs_status_t rocs_glm_fm_projection(const rocs_plan_t* plan, rocs_dtype_t dtype
                        g_path.load() == ROCS_PATH_AUTO, (cudaStream_t)stream_);
 }
 
+rocs_status_t rocs_group_norm(rocs_dtype_t dtype, rocs_norm_t kind, int64_t M, int32_t d, const void* X,
+                              int64_t ld_x, const void* gamma, const void* beta, float eps, void* Y, int64_t ld_y,
+                              void* stream_) {
+  if ((dtype != ROCS_BF16 && dtype != ROCS_F32) || (kind != ROCS_NORM_LAYER && kind != ROCS_NORM_RMS))
+    return ROCS_ERR_INVALID_ARG;
+  if (M < 0 || d <= 0 || ld_x < d || ld_y < d || !(eps >= 0.f)) return ROCS_ERR_INVALID_ARG;
+  if (M > 0 && (!X || !Y)) return ROCS_ERR_INVALID_ARG;
+  const int64_t es = (int64_t)elem_size(dtype);
+  if (!aligned16(X) || !aligned16(Y) || !aligned16(gamma) || !aligned16(beta) || (ld_x * es) % 16 != 0 ||
+      (ld_y * es) % 16 != 0)
+    return ROCS_ERR_ALIGNMENT;
+  return group_norm(dtype, (int)kind, M, d, X, ld_x, gamma, beta, eps, Y, ld_y, (cudaStream_t)stream_);
+}
+
 rocs_status_t rocs_last_device_status(uint32_t* detail_host) {
   uint32_t* word = device_status_word();
   if (!word) return ROCS_ERR_CUDA;

@@ -91,6 +91,10 @@ rocs_status_t simt_glm(rocs_dtype_t dt, const rocs_plan* plan, int32_t n_r, int3
                        void* YR, void* YC, void* OR_, void* OC, float* zr_workspace,
                        cudaStream_t stream);
 
+// ---- group-local normalisation (Eq. 7): group_norm.cu -------------------------------------
+rocs_status_t group_norm(rocs_dtype_t dt, int kind, int64_t M, int32_t d, const void* X, int64_t ld_x,
+                         const void* gamma, const void* beta, float eps, void* Y, int64_t ld_y, cudaStream_t stream);
+
 // ---- projected factorization machine: fm_projection.cu ----------------------------------
 // F = G P on the request-once form; tt_workspace [R, k, d] fp32 receives P_R^T X^R per request.
 // allow_fast: use the bf16 streaming kernel for the candidate side where the shape allows it.
