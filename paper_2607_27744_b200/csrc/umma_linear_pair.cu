@@ -25,8 +25,8 @@ constexpr int kEpiWarps = 8;
 constexpr int kABytes = BM * BK * 2;         // 16 KB: this CTA's rows of X
 constexpr int kBBytes = (BN / 2) * BK * 2;   // 16 KB: this CTA's half of the weight tile
 constexpr int kStageBytes = kABytes + kBBytes;
-constexpr int kStages = 5;
-constexpr int kStagingBytes = kEpiWarps * 8192;
+constexpr int kStages = 6;
+constexpr int kStagingBytes = kEpiWarps * 4096;  // one 32-row x 128-byte box per warp, used by both column chunks
 constexpr int kSmemBytes = kStages * kStageBytes + kStagingBytes + 512 + 1024;
 constexpr uint32_t kStatusPair = 0x600;
 
@@ -142,7 +142,7 @@ linear_pair_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_const
     // ------------------------------ epilogue (both CTAs) ------------------------------------
     const int q = warp % 4;
     const int half = (warp - 2) / 4;
-    uint8_t* my_stage = staging + (warp - 2) * 8192;
+    uint8_t* my_stage = staging + (warp - 2) * 4096;
     const uint32_t tmem_empty_leader[2] = {map_to_cta(smem_u32(&tmem_empty[0]), 0),
                                            map_to_cta(smem_u32(&tmem_empty[1]), 0)};
     uint32_t lt = 0;
@@ -183,7 +183,11 @@ linear_pair_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_const
 #pragma unroll
           for (int i = 0; i < 64; ++i) f[i] = fmaxf(f[i], 0.f);
         }
-        uint8_t* row_ptr = my_stage + c * 4096 + lane * 128;
+        if (c == 1) {  // the store of the first chunk has finished reading the box
+          if (lane == 0) tma_store_wait_read<0>();
+          __syncwarp();
+        }
+        uint8_t* row_ptr = my_stage + lane * 128;
 #pragma unroll
         for (int j = 0; j < 8; ++j) {
           uint4 w;
@@ -197,15 +201,12 @@ linear_pair_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_const
           w.w = *reinterpret_cast<uint32_t*>(&h3);
           *reinterpret_cast<uint4*>(row_ptr + ((j ^ (lane & 7)) << 4)) = w;
         }
-      }
-      fence_proxy_async_smem();
-      __syncwarp();
-      if (lane == 0) {
-#pragma unroll
-        for (int c = 0; c < 2; ++c)
-          if (n0 + half * 128 + c * 64 < p.d_out && (int64_t)m0 + q * 32 < p.M)
-            tma_store_2d(&map_y, my_stage + c * 4096, n0 + half * 128 + c * 64, m0 + q * 32);
-        tma_store_commit();
+        fence_proxy_async_smem();
+        __syncwarp();
+        if (lane == 0) {
+          if (col0 < p.d_out && (int64_t)m0 + q * 32 < p.M) tma_store_2d(&map_y, my_stage, col0, m0 + q * 32);
+          tma_store_commit();
+        }
       }
     }
     if (lane == 0) tma_store_wait_all<0>();
