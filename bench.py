@@ -277,6 +277,19 @@ def run_rocs(args):
 
     t_plan_in, t_l1, t_l2, t_l3 = span(0, 1), span(1, 2), span(2, 3), span(3, 4)
 
+    def span_median(ms_, a, b):
+        return float(np.median([m[a].elapsed_time(m[b]) for m in ms_])) * 1e-3
+
+    medians = [span_median(marks, a, a + 1) for a in (1, 2, 3)]
+    # the same step on ONE buffer set (inputs and weights stay in L2 as far as they fit): "warm" figures
+    warm_marks = [[torch.cuda.Event(enable_timing=True) for _ in range(5)] for _ in range(30)]
+    for i in range(3):
+        step(0)
+    for wm in warm_marks:
+        step(0, marks=wm)
+    torch.cuda.synchronize()
+    warm = [span_median(warm_marks, a, a + 1) for a in (1, 2, 3)]
+
     def time_call(fn, reps=20):
         for i in range(3):
             fn(i)
@@ -328,6 +341,9 @@ def run_rocs(args):
     t_mat = time_call(lambda i: materialised_linear(torch, XR_sets[i % N_SETS], XC_sets[i % N_SETS], W1, counts_dev), reps=10)
     layers[0]["materialised_broadcast_gpu_us"] = t_mat * 1e6
     layers[0]["speedup_vs_materialised"] = t_mat / t_l1
+    for lay, med, w in zip(layers, medians, warm):
+        lay["us_median"] = med * 1e6            # median over the timed steps (rotating sets: cold L2)
+        lay["us_warm_l2"] = w * 1e6             # median of 30 steps on one buffer set
 
     # ---- attention and interaction kernels on their own workloads ----------------------------
     extra = []
