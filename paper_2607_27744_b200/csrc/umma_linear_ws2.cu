@@ -169,11 +169,12 @@ linear_ws2_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_consta
       }
     }
   } else if (warp == 1) {
-    // ------------------------------ MMA issuer (leader CTA only) ---------------------------
-    if (rank == 0) {
+    // ------------------------------ MMA issuer (leader CTA only): a single thread -----------
+    if (rank == 0 && lane == 0) {
       constexpr uint32_t idesc = umma_idesc_bf16(2 * BM, BN, false, false);
       uint32_t it = 0, lt = 0;
       bool ok = mbar_wait(w_full, 0, abort_flag, p.status, kStatusWs2 | 6);
+      const uint64_t b_desc0 = smem_desc_sw128(smem_u32(w_smem), 1024, 16);
       for (int32_t st = group; st < super_tiles && ok; st += p.groups, ++lt) {
         const uint32_t acc = lt & 1;
         if (!mbar_wait(&tmem_empty[acc], ((lt >> 1) & 1) ^ 1, abort_flag, p.status, kStatusWs2 | 2)) { ok = false; break; }
@@ -183,20 +184,16 @@ linear_ws2_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_consta
           const int s = it % p.a_stages;
           if (!mbar_wait(&a_full[s], (it / p.a_stages) & 1, abort_flag, p.status, kStatusWs2 | 3)) { ok = false; break; }
           tc_fence_after_sync();
-          if (lane == 0) {
-            const uint64_t a_desc = smem_desc_sw128(smem_u32(a_smem + s * kAStageBytes), 1024, 16);
-            const uint64_t b_desc = smem_desc_sw128(smem_u32(w_smem + kb * kWBlockBytes), 1024, 16);
+          const uint64_t a_desc = smem_desc_sw128(smem_u32(a_smem + s * kAStageBytes), 1024, 16);
+          const uint64_t b_desc = b_desc0 + kb * (kWBlockBytes >> 4);
 #pragma unroll
-            for (int k = 0; k < BK / 16; ++k)
-              umma_ss_pair(d_tmem, a_desc + 2 * k, b_desc + 2 * k, idesc, (kb | k) != 0 ? 1u : 0u);
-            umma_commit_pair(&a_empty[s], 3);  // frees the stage in both CTAs
-          }
-          __syncwarp();
+          for (int k = 0; k < BK / 16; ++k)
+            umma_ss_pair(d_tmem, a_desc + 2 * k, b_desc + 2 * k, idesc, (kb | k) != 0 ? 1u : 0u);
+          umma_commit_pair(&a_empty[s], 3);  // frees the stage in both CTAs
         }
-        if (ok && lane == 0) umma_commit_pair(&tmem_full[acc], 3);
-        __syncwarp();
+        if (ok) umma_commit_pair(&tmem_full[acc], 3);
       }
-      if (!ok && lane == 0) {
+      if (!ok) {
         umma_commit_pair(drain, 1);
         const uint64_t t0 = globaltimer_ns();
         while (!mbar_try_wait(drain, 0) && globaltimer_ns() - t0 < kWaitLimitNs) {}
