@@ -216,12 +216,21 @@ fm_candidate_mma_kernel(const __grid_constant__ CUtensorMap map_xc, const FmPara
     float tfrag[kPairs][2][4];  // T^T of the cached request in step-1 accumulator layout
     int32_t cached_req = -1;
     uint32_t it = 0;
+    // the request of this warp's candidate, fetched one tile ahead of its use (the load would
+    // otherwise sit on every candidate's critical path)
+    int32_t r_next = 0;
+    if (tile_begin < tile_end && (int64_t)tile_begin * kTileCands + warp < p.N)
+      r_next = p.row2req[(int64_t)tile_begin * kTileCands + warp];
     for (int32_t t = tile_begin; t < tile_end; ++t, ++it) {
       const int s = it % STAGES;
+      const int32_t r = r_next;
+      {
+        const int64_t cand_next = (int64_t)(t + 1) * kTileCands + warp;
+        if (t + 1 < tile_end && cand_next < p.N) r_next = p.row2req[cand_next];
+      }
       if (!mbar_wait(&full[s], (it / STAGES) & 1, abort_flag, p.status, kStatusFm | 2)) break;
       const int64_t cand = (int64_t)t * kTileCands + warp;
       if (cand < p.N) {
-        const int32_t r = p.row2req[cand];
         if (r != cached_req) {
           if (cached_req < 0) griddep_wait();  // TT comes from the request kernel launched just before
           cached_req = r;
