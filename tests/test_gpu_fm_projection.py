@@ -42,7 +42,7 @@ def test_config1_fp32_every_element():
 
 @pytest.mark.parametrize("path", PATHS)
 @pytest.mark.parametrize("k", [8, 16])
-@pytest.mark.parametrize("d_emb", [64, 128, 256])
+@pytest.mark.parametrize("d_emb", [64, 128, 192, 256])
 def test_bf16_ragged_segments_and_tail_tile(path, k, d_emb):
     # empty requests, single candidates, segments that straddle the 8-candidate tiles, N % 8 != 0
     co = wl.offsets_from_counts([1, 0, 9, 8, 33, 7, 0, 133])
@@ -57,6 +57,12 @@ def test_bf16_shapes_outside_the_streaming_kernel(path):
     assert _run(cfg, co, 12, path=path) <= tol_for("bf16")
     cfg = wl.CONFIGS[4].with_(R=3, n_r=8, n_c=16, d_emb=32)
     assert _run(cfg, co, 16, path=path) <= tol_for("bf16")
+
+
+def test_wide_request_group():
+    co = wl.offsets_from_counts([3, 70, 5])
+    cfg = wl.CONFIGS[4].with_(R=3, n_r=64, d_emb=256)
+    assert _run(cfg, co, 16) <= tol_for("bf16")
 
 
 def test_many_tiles_per_cta():

@@ -18,7 +18,7 @@ def _inputs(M, d, dtype, seed):
 
 
 @pytest.mark.parametrize("kind", [rocs.NORM_LAYER, rocs.NORM_RMS])
-@pytest.mark.parametrize("dtype,d", [("bf16", 256), ("bf16", 1024), ("bf16", 768), ("bf16", 2048), ("bf16", 4096),
+@pytest.mark.parametrize("dtype,d", [("bf16", 256), ("bf16", 1024), ("bf16", 768), ("bf16", 1536), ("bf16", 2048), ("bf16", 4096),
                                      ("bf16", 40), ("f32", 128), ("f32", 96), ("f32", 1024)])
 def test_rows_against_the_oracle(kind, dtype, d):
     x, gamma, beta = _inputs(1237, d, dtype, d % 7)
