@@ -141,8 +141,8 @@ def run_reference(args):
         return
     data = host_inputs(wl.CONFIGS[2])
     probe_rate, threads, _ = oracle_mlp_rate(64, data)
-    budget_s = min(8.0, 120.0 / max(1, args.steps + args.warmup))   # whole run within a few minutes
-    per_step = int(max(8, min(4096, probe_rate * budget_s)))
+    seconds_per_step = min(8.0, 120.0 / max(1, args.steps + args.warmup))   # whole run within a few minutes
+    per_step = int(max(8, min(4096, probe_rate * seconds_per_step)))
     for _ in range(args.warmup):
         oracle_mlp_rate(per_step, data)
     t0 = time.perf_counter()
