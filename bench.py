@@ -341,6 +341,11 @@ def run_rocs(args):
     t_mat = time_call(lambda i: materialised_linear(torch, XR_sets[i % N_SETS], XC_sets[i % N_SETS], W1, counts_dev), reps=10)
     layers[0]["materialised_broadcast_gpu_us"] = t_mat * 1e6
     layers[0]["speedup_vs_materialised"] = t_mat / t_l1
+    # library GEMM (torch.matmul -> cuBLAS) on the plain layers, same buffers: a reference point
+    t_lib2 = time_call(lambda i: torch.relu_(torch.matmul(h1[i % N_SETS], W2.t())), reps=10)
+    t_lib3 = time_call(lambda i: torch.matmul(h2[i % N_SETS], W3.t()), reps=10)
+    layers[1]["library_gemm_relu_us"] = t_lib2 * 1e6
+    layers[2]["library_gemm_us"] = t_lib3 * 1e6
     for lay, med, w in zip(layers, medians, warm):
         lay["us_median"] = med * 1e6            # median over the timed steps (rotating sets: cold L2)
         lay["us_warm_l2"] = w * 1e6             # median of 30 steps on one buffer set
