@@ -67,11 +67,13 @@ rocs_status_t plan_tiles(const rocs_plan* plan, int32_t cands_per_tile, cudaStre
   return ROCS_OK;
 }
 
-rocs_status_t plan_dca_items(const rocs_plan* plan, int32_t cands_per_tile, int32_t heads, cudaStream_t stream,
-                             DcaItemList* out) {
-  if (cands_per_tile < 1 || cands_per_tile > 32767 || heads < 1 || heads > 65535) return ROCS_ERR_INVALID_ARG;
+rocs_status_t plan_dca_items(const rocs_plan* plan, int32_t cands_per_tile, int32_t heads, int32_t tiles_per_item,
+                             cudaStream_t stream, DcaItemList* out) {
+  if (cands_per_tile < 1 || cands_per_tile > 32767 || heads < 1 || heads > 65535 || tiles_per_item < 1 ||
+      tiles_per_item > 2)
+    return ROCS_ERR_INVALID_ARG;
   std::lock_guard<std::mutex> lock(plan->mu);
-  const int64_t key = (int64_t)cands_per_tile * 65536 + heads;
+  const int64_t key = ((int64_t)cands_per_tile * 65536 + heads) * 2 + (tiles_per_item - 1);
   auto it = plan->dca_items.find(key);
   if (it != plan->dca_items.end()) {
     *out = it->second;
@@ -82,9 +84,9 @@ rocs_status_t plan_dca_items(const rocs_plan* plan, int32_t cands_per_tile, int3
     const int32_t c_begin = plan->offsets_host[r], c_end = plan->offsets_host[r + 1];
     if (c_begin == c_end) continue;
     for (int32_t h = 0; h < heads; ++h)
-      for (int32_t c = c_begin; c < c_end; c += 2 * cands_per_tile) {
+      for (int32_t c = c_begin; c < c_end; c += tiles_per_item * cands_per_tile) {
         const int32_t a = std::min(cands_per_tile, c_end - c);
-        const int32_t b = std::min(cands_per_tile, c_end - c - a);
+        const int32_t b = tiles_per_item == 2 ? std::min(cands_per_tile, c_end - c - a) : 0;
         host.push_back(DcaItem{r, c, (int16_t)a, (int16_t)b, h});
       }
   }

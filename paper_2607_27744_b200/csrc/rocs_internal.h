@@ -51,7 +51,7 @@ struct rocs_plan {
   std::vector<int32_t> offsets_host;      // [R+1]
   mutable std::mutex mu;
   mutable std::map<int32_t, rocs::TileList> tiles;  // key: candidates per tile
-  mutable std::map<int64_t, rocs::DcaItemList> dca_items;  // key: candidates per tile * 65536 + heads
+  mutable std::map<int64_t, rocs::DcaItemList> dca_items;  // key: (candidates per tile * 65536 + heads) * 2 + tiles per item - 1
   int device = 0;
   cudaStream_t stream = nullptr;  // stream the plan was created on; its memory is freed there
 };
@@ -72,9 +72,10 @@ inline size_t round_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 rocs_status_t plan_tiles(const rocs_plan* plan, int32_t cands_per_tile, cudaStream_t stream,
                          TileList* out);
 
-// Work items for the attention kernel, ordered request, head, tile pair; cached in the plan.
-rocs_status_t plan_dca_items(const rocs_plan* plan, int32_t cands_per_tile, int32_t heads, cudaStream_t stream,
-                             DcaItemList* out);
+// Work items for the attention kernel, ordered request, head, tile (or tile pair when tiles_per_item is 2);
+// cached in the plan.
+rocs_status_t plan_dca_items(const rocs_plan* plan, int32_t cands_per_tile, int32_t heads, int32_t tiles_per_item,
+                             cudaStream_t stream, DcaItemList* out);
 
 // ---- general (CUDA-core) kernels: simt_kernels.cu -------------------------------------
 // Y[i, :] = act(add[row2req ? row2req[i] : -, :] + X[i, :] W^T + bias).  out_f32 selects an

@@ -43,17 +43,17 @@ constexpr int DH = 64;            // head dimension handled here (128-byte rows)
 constexpr int BQ = 128;           // query rows per tile
 constexpr int BKV = 128;          // keys per block
 constexpr int kSoftmaxWarps = 16; // 8 per side
-constexpr int kControlWarp0 = kSoftmaxWarps;   // warp 16: TMA producer, 17 and 18: MMA issuers of sides A and B, 19 idle
+constexpr int kControlWarp0 = kSoftmaxWarps;   // warps 16, 19: TMA producers of sides A, B; 17, 18: their MMA issuers
 constexpr int kThreads = (kSoftmaxWarps + 4) * 32;
-constexpr int kKvStages = 4;
-constexpr int kQSlots = 2;        // Q buffers per side: the producer runs one item ahead
+constexpr int kKvStages = 3;        // per side
+constexpr int kQSlots = 1;         // Q buffers per side (freed when the item's last S is issued, a block before its end)
 constexpr int kTmemCols = 512;
 constexpr int kQBytes = BQ * DH * 2;            // 16 KB
 constexpr int kKBytes = BKV * DH * 2;           // 16 KB
 constexpr int kKvStageBytes = 2 * kKBytes;      // K block + V block
 constexpr int kXchgBytes = 2 * 2 * BQ * 4;  // partial sums of the two halves of a row [side][half][row]
-constexpr int kNumBarriers = 2 * kQSlots + 2 * kKvStages + 8 + 8 + 2;
-constexpr int kSmemBytes = kQSlots * 2 * kQBytes + kKvStages * kKvStageBytes + kXchgBytes + kNumBarriers * 8 + 16;
+constexpr int kNumBarriers = 2 * (2 * kQSlots + 2 * kKvStages) + 8 + 8 + 2;
+constexpr int kSmemBytes = 2 * (kQSlots * kQBytes + kKvStages * kKvStageBytes) + kXchgBytes + kNumBarriers * 8 + 16;
 constexpr float kRescaleThreshold = 8.f;  // log2 units
 constexpr uint32_t kStatusDca = 0x400;
 constexpr int kSideTmemStride = 256;
@@ -75,9 +75,13 @@ struct DcaParams {
 };
 
 __device__ __forceinline__ float ex2(float x) {
+#ifdef ROCS_DCA_PROBE_NOEXP
+  return x * 0.001f;  // timing probe only: wrong results
+#else
   float y;
   asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
   return y;
+#endif
 }
 
 // Packed fp32 pairs (one instruction for two lanes of arithmetic) and the three-input maximum.
@@ -133,7 +137,7 @@ __device__ __forceinline__ void tmem_st_32x32b_x32(uint32_t taddr, const uint32_
 // One query row of one head, 32 of its 64 output columns, in plain fp32 with the row's true maximum as
 // reference: q and k point at the head's 64 values of the row / of the request's first key, v at the
 // 32 columns wanted; consecutive keys are `stride` elements apart.
-__device__ __noinline__ void row_by_hand(const __nv_bfloat16* q, const __nv_bfloat16* k, const __nv_bfloat16* v,
+__device__ __forceinline__ void row_by_hand(const __nv_bfloat16* q, const __nv_bfloat16* k, const __nv_bfloat16* v,
                                          int32_t stride, int32_t L, float scale_log2e, __nv_bfloat16* out) {
   auto score = [&](int32_t j) {
     float s = 0.f;
@@ -174,14 +178,14 @@ __global__ void __launch_bounds__(kThreads, 1)
 dca_umma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
                 const __grid_constant__ CUtensorMap map_v, const DcaParams p) {
   extern __shared__ __align__(1024) uint8_t smem[];     // swizzled operand tiles need 1024-byte alignment
-  uint8_t* q_smem = smem;                                // [slots][2 sides][128][64] bf16
-  uint8_t* kv_smem = q_smem + kQSlots * 2 * kQBytes;     // [stages][K 16 KB | V 16 KB]
-  float* l_x = reinterpret_cast<float*>(kv_smem + kKvStages * kKvStageBytes);  // [2 sides][2 halves][128]
-  uint64_t* q_full = reinterpret_cast<uint64_t*>(l_x + 2 * 2 * BQ);  // [slots]
-  uint64_t* q_empty = q_full + kQSlots;      // [slots]
-  uint64_t* kv_full = q_empty + kQSlots;
-  uint64_t* kv_empty = kv_full + kKvStages;
-  uint64_t* s_full = kv_empty + kKvStages;   // [2]
+  uint8_t* q_smem = smem;                                // [2 sides][slots][128][64] bf16
+  uint8_t* kv_smem = q_smem + 2 * kQSlots * kQBytes;     // [2 sides][stages][K 16 KB | V 16 KB]
+  float* l_x = reinterpret_cast<float*>(kv_smem + 2 * kKvStages * kKvStageBytes);  // [2 sides][2 halves][128]
+  uint64_t* q_full = reinterpret_cast<uint64_t*>(l_x + 2 * 2 * BQ);  // [2 sides][slots]
+  uint64_t* q_empty = q_full + 2 * kQSlots;      // [2][slots]
+  uint64_t* kv_full = q_empty + 2 * kQSlots;     // [2][stages]
+  uint64_t* kv_empty = kv_full + 2 * kKvStages;  // [2][stages]
+  uint64_t* s_full = kv_empty + 2 * kKvStages;   // [2]
   uint64_t* s_empty = s_full + 2;            // [2]
   uint64_t* p_full = s_empty + 2;            // [2]
   uint64_t* o_full = p_full + 2;             // [2]
@@ -197,13 +201,13 @@ dca_umma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
   }
 
   if (threadIdx.x == 0) {
-    for (int x = 0; x < kQSlots; ++x) {
+    for (int x = 0; x < 2 * kQSlots; ++x) {
       mbar_init(&q_full[x], 1);
-      mbar_init(&q_empty[x], 2);
+      mbar_init(&q_empty[x], 1);
     }
-    for (int s = 0; s < kKvStages; ++s) {
+    for (int s = 0; s < 2 * kKvStages; ++s) {
       mbar_init(&kv_full[s], 1);
-      mbar_init(&kv_empty[s], 2);
+      mbar_init(&kv_empty[s], 1);
     }
     for (int x = 0; x < 2; ++x) {
       mbar_init(&s_full[x], 1);
@@ -227,36 +231,41 @@ dca_umma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
   const uint32_t tmem_base = *tmem_ptr;
   const int32_t row_width = p.H * DH;  // elements per query / key row over all heads
 
-  if (warp >= kControlWarp0) {
-  if (warp == kControlWarp0) {
-    // ------------------------------ TMA producer ------------------------------------------
+  // Each side is a stream of its own: items 2 b + side, 2 b + side + 2 grid, ... of CTA b.
+  const int32_t item0 = 2 * (int32_t)blockIdx.x, item_step = 2 * (int32_t)gridDim.x;
+
+  if (warp == kControlWarp0 || warp == kControlWarp0 + 3) {
+    // ------------------------------ TMA producers: one warp per side --------------------------
+    const int side = warp == kControlWarp0 ? 0 : 1;
     if (lane == 0) {
       prefetch_tensormap(&map_q);
       prefetch_tensormap(&map_k);
       prefetch_tensormap(&map_v);
+      uint64_t* qf = q_full + side * kQSlots;
+      uint64_t* qe = q_empty + side * kQSlots;
+      uint64_t* kf = kv_full + side * kKvStages;
+      uint64_t* ke = kv_empty + side * kKvStages;
+      uint8_t* kv_side = kv_smem + side * kKvStages * kKvStageBytes;
       uint32_t kv_it = 0, n_work = 0;
       bool ok = true;
-      for (int32_t i = blockIdx.x; i < p.num_items && ok; i += gridDim.x) {
+      for (int32_t i = item0 + side; i < p.num_items && ok; i += item_step) {
         const DcaItem item = p.items[i];
         const int32_t s0 = p.seq_offsets[item.req];
         const int32_t L = p.seq_offsets[item.req + 1] - s0;
         if (L == 0) continue;  // nobody touches a barrier for an item without keys
         const uint32_t slot = n_work % kQSlots;
-        if (!mbar_wait_paced(&q_empty[slot], ((n_work / kQSlots) & 1) ^ 1, abort_flag, p.status, kStatusDca | 1)) { ok = false; break; }
+        if (!mbar_wait_paced(&qe[slot], ((n_work / kQSlots) & 1) ^ 1, abort_flag, p.status, kStatusDca | 1)) { ok = false; break; }
         ++n_work;
-        const int32_t sides = item.count_b > 0 ? 2 : 1;
-        uint8_t* qs = q_smem + slot * 2 * kQBytes;
-        mbar_expect_tx(&q_full[slot], sides * kQBytes);
-        tma_load_2d(qs, &map_q, &q_full[slot], item.head * DH, item.cand0 * p.n_q);
-        if (sides == 2) tma_load_2d(qs + kQBytes, &map_q, &q_full[slot], item.head * DH, (item.cand0 + item.count_a) * p.n_q);
+        mbar_expect_tx(&qf[slot], kQBytes);
+        tma_load_2d(q_smem + (side * kQSlots + slot) * kQBytes, &map_q, &qf[slot], item.head * DH, item.cand0 * p.n_q);
         const int32_t nblk = (L + BKV - 1) / BKV;
         for (int32_t j = 0; j < nblk; ++j, ++kv_it) {
           const int s = kv_it % kKvStages;
-          if (!mbar_wait_paced(&kv_empty[s], ((kv_it / kKvStages) & 1) ^ 1, abort_flag, p.status, kStatusDca | 2)) { ok = false; break; }
-          uint8_t* st = kv_smem + s * kKvStageBytes;
-          mbar_expect_tx(&kv_full[s], kKvStageBytes);
-          tma_load_2d(st, &map_k, &kv_full[s], item.head * DH, s0 + j * BKV);
-          tma_load_2d(st + kKBytes, &map_v, &kv_full[s], item.head * DH, s0 + j * BKV);
+          if (!mbar_wait_paced(&ke[s], ((kv_it / kKvStages) & 1) ^ 1, abort_flag, p.status, kStatusDca | 2)) { ok = false; break; }
+          uint8_t* st = kv_side + s * kKvStageBytes;
+          mbar_expect_tx(&kf[s], kKvStageBytes);
+          tma_load_2d(st, &map_k, &kf[s], item.head * DH, s0 + j * BKV);
+          tma_load_2d(st + kKBytes, &map_v, &kf[s], item.head * DH, s0 + j * BKV);
         }
       }
       if (!ok) {
@@ -265,15 +274,20 @@ dca_umma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
           const uint32_t n_issued = kv_it / kKvStages + (((int)(kv_it % kKvStages) > s) ? 1 : 0);
           if (n_issued == 0) continue;
           const uint64_t t0 = globaltimer_ns();
-          while (!mbar_try_wait(&kv_full[s], (n_issued - 1) & 1) && globaltimer_ns() - t0 < kWaitLimitNs) {}
+          while (!mbar_try_wait(&kf[s], (n_issued - 1) & 1) && globaltimer_ns() - t0 < kWaitLimitNs) {}
         }
       }
     }
-  } else if (warp <= kControlWarp0 + 2) {
+  } else if (warp >= kControlWarp0) {
     // ------------------------------ MMA issuers: one warp per side ---------------------------
     const int side = warp - (kControlWarp0 + 1);
     constexpr uint32_t idesc_s = umma_idesc_bf16(BQ, BKV, false, false);  // S = Q K^T, both K-major
     constexpr uint32_t idesc_o = umma_idesc_bf16(BQ, DH, false, true);    // O = P V, V is MN-major
+    uint64_t* qf = q_full + side * kQSlots;
+    uint64_t* qe = q_empty + side * kQSlots;
+    uint64_t* kf = kv_full + side * kKvStages;
+    uint64_t* ke = kv_empty + side * kKvStages;
+    uint8_t* kv_side = kv_smem + side * kKvStages * kKvStageBytes;
     uint32_t kv_it = 0, n_work = 0;           // n_work: items that had keys (phase of q_full)
     uint32_t cnt_p = 0, cnt_se = 0;           // phases of p_full and s_empty of this side
     bool ok = true;
@@ -281,17 +295,19 @@ dca_umma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
     int tr_blk = 0;
 #endif
     const uint32_t t_s = tmem_base + side * kSideTmemStride;
-    auto issue_s = [&](int stage, uint32_t slot) {
-      const uint64_t a_desc = smem_desc_sw128(smem_u32(q_smem + (slot * 2 + side) * kQBytes), 1024, 16);
-      const uint64_t b_desc = smem_desc_sw128(smem_u32(kv_smem + stage * kKvStageBytes), 1024, 16);
+    // Descriptors are formed by the whole warp ahead of the barrier waits; the elected lane then only
+    // issues the products.
+    auto desc_q = [&](uint32_t slot) { return smem_desc_sw128(smem_u32(q_smem + (side * kQSlots + slot) * kQBytes), 1024, 16); };
+    auto desc_k = [&](int stage) { return smem_desc_sw128(smem_u32(kv_side + stage * kKvStageBytes), 1024, 16); };
+    auto desc_v = [&](int stage) { return smem_desc_sw128(smem_u32(kv_side + stage * kKvStageBytes + kKBytes), 1024, 16); };
+    auto issue_s = [&](uint64_t a_desc, uint64_t b_desc) {
 #pragma unroll
       for (int k = 0; k < DH / 16; ++k) umma_ss(t_s, a_desc + 2 * k, b_desc + 2 * k, idesc_s, k != 0 ? 1u : 0u);
       umma_commit(&s_full[side]);
     };
-    auto issue_pv = [&](int stage, bool first_block) {
+    auto issue_pv = [&](uint64_t b_desc, bool first_block) {
       // P: 16 keys = 8 columns of bf16 pairs in tensor memory
       // V: rows are keys (K), 128 bytes = 64 head dims (N): 16 keys = 2048 bytes further on
-      const uint64_t b_desc = smem_desc_sw128(smem_u32(kv_smem + stage * kKvStageBytes + kKBytes), 1024, 16);
 #pragma unroll
       for (int k = 0; k < BKV / 16; ++k)
         umma_ts(t_s + kOColOffset, t_s + kPColOffset + k * 8, b_desc + k * (16 * 128 / 16), idesc_o,
@@ -301,48 +317,40 @@ dca_umma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
     // The last block of a sequence may reach past it into the next request's rows (or past the
     // tensor, where TMA fills zeros).  Scores of such keys are masked to -inf by the softmax warps,
     // so P is exactly 0 there; the V rows are zeroed here so that 0 x (Inf or NaN of a foreign
-    // request) cannot reach this request's output.  Both issuers write the same zeros, each before
-    // its own product reads the tile.
+    // request) cannot reach this request's output.
     auto zero_v_tail = [&](int stage, int32_t valid) {
-      uint8_t* v = kv_smem + stage * kKvStageBytes + kKBytes;
+      uint8_t* v = kv_side + stage * kKvStageBytes + kKBytes;
       for (int idx = valid * 8 + lane; idx < BKV * 8; idx += 32)
         *reinterpret_cast<uint4*>(v + idx * 16) = make_uint4(0u, 0u, 0u, 0u);
       fence_proxy_async_smem();
       __syncwarp();
     };
-    for (int32_t i = blockIdx.x; i < p.num_items && ok; i += gridDim.x) {
+    for (int32_t i = item0 + side; i < p.num_items && ok; i += item_step) {
       const DcaItem item = p.items[i];
       const int32_t L = p.seq_offsets[item.req + 1] - p.seq_offsets[item.req];
       if (L == 0) continue;
       const int32_t nblk = (L + BKV - 1) / BKV;
       const int32_t tail_valid = L - (nblk - 1) * BKV;  // keys of the last block that exist
       const uint32_t slot = n_work % kQSlots;
-      if (!mbar_wait_paced(&q_full[slot], (n_work / kQSlots) & 1, abort_flag, p.status, kStatusDca | 3)) { ok = false; break; }
+      if (!mbar_wait_paced(&qf[slot], (n_work / kQSlots) & 1, abort_flag, p.status, kStatusDca | 3)) { ok = false; break; }
       ++n_work;
-      if (side == 1 && item.count_b == 0) {
-        // no second tile: hand every buffer back in step with the other issuer
-        if (lane == 0) mbar_arrive(&q_empty[slot]);
-        for (int32_t j = 0; j < nblk; ++j, ++kv_it) {
-          if (!mbar_wait_paced(&kv_full[kv_it % kKvStages], (kv_it / kKvStages) & 1, abort_flag, p.status, kStatusDca | 4)) { ok = false; break; }
-          if (lane == 0) mbar_arrive(&kv_empty[kv_it % kKvStages]);
-        }
-        continue;
-      }
       // first key block (the S tile was drained at the end of the previous item)
-      if (!mbar_wait_paced(&kv_full[kv_it % kKvStages], (kv_it / kKvStages) & 1, abort_flag, p.status, kStatusDca | 4)) { ok = false; break; }
+      if (!mbar_wait_paced(&kf[kv_it % kKvStages], (kv_it / kKvStages) & 1, abort_flag, p.status, kStatusDca | 4)) { ok = false; break; }
       if (nblk == 1 && tail_valid < BKV) zero_v_tail(kv_it % kKvStages, tail_valid);
       tc_fence_after_sync();
+      const uint64_t dq = desc_q(slot);
       if (lane == 0) {
-        issue_s(kv_it % kKvStages, slot);
-        if (nblk == 1) umma_commit(&q_empty[slot]);
+        issue_s(dq, desc_k(kv_it % kKvStages));
+        if (nblk == 1) umma_commit(&qe[slot]);
       }
       __syncwarp();
       for (int32_t j = 0; j < nblk && ok; ++j, ++kv_it) {
         const int stage = kv_it % kKvStages;
         const int next_stage = (kv_it + 1) % kKvStages;
+        const uint64_t dk_next = desc_k(next_stage), dv = desc_v(stage);
         TRACE_EV(2 + side, 0);
         if (j + 1 < nblk) {
-          if (!mbar_wait_paced(&kv_full[next_stage], ((kv_it + 1) / kKvStages) & 1, abort_flag, p.status, kStatusDca | 5)) { ok = false; break; }
+          if (!mbar_wait_paced(&kf[next_stage], ((kv_it + 1) / kKvStages) & 1, abort_flag, p.status, kStatusDca | 5)) { ok = false; break; }
           TRACE_EV(2 + side, 1);
           if (j + 2 == nblk && tail_valid < BKV) zero_v_tail(next_stage, tail_valid);
         }
@@ -353,20 +361,20 @@ dca_umma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
         if (j + 1 < nblk) {
           tc_fence_after_sync();
           if (lane == 0) {
-            issue_s(next_stage, slot);
-            if (j + 2 == nblk) umma_commit(&q_empty[slot]);  // last S of the item: Q slot is free
+            issue_s(dq, dk_next);
+            if (j + 2 == nblk) umma_commit(&qe[slot]);  // last S of the item: Q slot is free
           }
           __syncwarp();
           TRACE_EV(2 + side, 3);
         }
-        // P_j of this side is in tensor memory (and O has been rescaled if it had to be)
+        // P_j of this side is in tensor memory
         if (!mbar_wait_paced(&p_full[side], cnt_p & 1, abort_flag, p.status, kStatusDca | 6)) { ok = false; break; }
         ++cnt_p;
         TRACE_EV(2 + side, 4);
         tc_fence_after_sync();
         if (lane == 0) {
-          issue_pv(stage, j == 0);
-          umma_commit(&kv_empty[stage]);  // K_j and V_j are no longer needed by this side
+          issue_pv(dv, j == 0);
+          umma_commit(&ke[stage]);  // K_j and V_j are no longer needed
         }
         __syncwarp();
         TRACE_EV(2 + side, 5);
@@ -380,7 +388,6 @@ dca_umma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
       const uint64_t t0 = globaltimer_ns();
       while (!mbar_try_wait(&drain[side], 0) && globaltimer_ns() - t0 < kWaitLimitNs) {}
     }
-  }
   } else {
     // ------------------------------ softmax warps ------------------------------------------
     const int sw = warp;
@@ -402,11 +409,11 @@ dca_umma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
 #else
 #define TRACE_SM(ev)
 #endif
-    for (int32_t i = blockIdx.x; i < p.num_items; i += gridDim.x) {
+    for (int32_t i = item0 + side; i < p.num_items; i += item_step) {
       const DcaItem item = p.items[i];
       const int32_t L = p.seq_offsets[item.req + 1] - p.seq_offsets[item.req];
-      const int32_t my_count = side == 0 ? item.count_a : item.count_b;
-      const int32_t cand_first = side == 0 ? item.cand0 : item.cand0 + item.count_a;
+      const int32_t my_count = item.count_a;
+      const int32_t cand_first = item.cand0;
       const int32_t rows_valid = my_count * p.n_q;
       const int32_t head = item.head;
       auto out_ptr = [&]() { return p.O + ((int64_t)cand_first * p.n_q + row) * row_width + head * DH + half * 32; };
@@ -588,7 +595,7 @@ rocs_status_t umma_dca(const rocs_plan* plan, int32_t n_q, int32_t H, int32_t dh
   (void)dh;
   if (plan->N == 0) return ROCS_OK;
   DcaItemList items;
-  rocs_status_t st = plan_dca_items(plan, BQ / n_q, H, stream, &items);
+  rocs_status_t st = plan_dca_items(plan, BQ / n_q, H, /*tiles_per_item=*/1, stream, &items);
   if (st != ROCS_OK) return st;
   if (items.num == 0) return ROCS_OK;
   const uint64_t width = (uint64_t)H * DH;
@@ -622,7 +629,7 @@ rocs_status_t umma_dca(const rocs_plan* plan, int32_t n_q, int32_t H, int32_t dh
   p.trace = (long long*)rocs_dca_trace_buffer;
 #endif
   ROCS_CUDA_TRY(cudaFuncSetAttribute(dca_umma_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes));
-  const int grid = std::min(items.num, sm_count_dca());  // one CTA per SM
+  const int grid = std::min((items.num + 1) / 2, sm_count_dca());  // one CTA per SM, two item streams per CTA
   dca_umma_kernel<<<grid, kThreads, kSmemBytes, stream>>>(map_q, map_k, map_v, p);
   ROCS_CUDA_TRY(cudaGetLastError());
   return ROCS_OK;
