@@ -1,30 +1,30 @@
 // Group-wise cross attention, candidate side (Eq. 13), with the request's K/V shared inside the
 // kernel (Section 4.3.1):  O[i,t,h,:] = softmax_j(scale <Q[i,t,h,:], K[r,j,h,:]>) V[r,j,h,:],  r = m_i.
 //
-// Candidates of one request are stacked in the tile M dimension: a work item is one head of up to
-// TWO 128-row query tiles (sides A and B) of the same request, so every 128-key block of K and V is
-// loaded once and used by 256 query rows.  K/V are addressed per request through seq_offsets;
-// nothing is replicated per candidate.
+// Candidates of one request are stacked in the tile M dimension: a work item is one head of one
+// 128-row query tile of a request; K/V are addressed per request through seq_offsets and read in
+// 128-key blocks, nothing is replicated per candidate (tiles of the same request and head are
+// consecutive items, so their K/V blocks are read from L2 at about the same time).
 //
-// One persistent CTA per SM, 20 warps:
-//   warp 16     TMA producer: Q tiles of the item (double buffered, one item ahead), then
-//               (K_j, V_j) blocks of 128 keys through a ring
-//   warps 17,18 tcgen05.mma issuers, one per side:  S_X = Q_X K_j^T (128x128x64, operands in shared
-//               memory) and O_X += P_X V_j (128x64x128, P read from tensor memory, V from shared memory)
-//   warps 0-15  softmax: 8 warps per side, TWO threads per query row, each owning 64 of the 128
-//               key columns of a block: S from TMEM into registers (one read), block maximum
-//               (the two halves of a row exchange theirs through shared memory), exp2 on scaled
-//               scores, fp32 partial sums, P rounded to bf16 and stored to tensor memory.
+// One persistent CTA per SM runs TWO independent item streams (sides A and B), 20 warps:
+//   warps 16,19 TMA producers of sides A, B: the Q tile of the item, then (K_j, V_j) blocks through a ring
+//   warps 17,18 tcgen05.mma issuers of sides A, B:  S = Q K_j^T (128x128x64, operands in shared memory)
+//               and O += P V_j (128x64x128, P read from tensor memory, V from shared memory)
+//   warps 0-15  softmax: 8 warps per side, TWO threads per query row, each owning 64 of the 128 key
+//               columns of a block: S from TMEM into registers (one read), exp2 on scaled scores,
+//               fp32 partial sums, P rounded to bf16 and stored to tensor memory.
 // Tensor memory per side (256 columns): S [0,128) fp32, P [128,192) bf16 pairs, O [192,256) fp32.
-// P has its own columns, so S_{j+1} is issued as soon as S_j sits in registers and the only wait
-// on P V_{j-1} comes after the exponentials of block j, just before P_j overwrites P_{j-1}: no
-// product and no hand-shake is on the softmax warps' critical path, they run back to back on the
-// exponential unit while the tensor pipe works one block ahead (S) and one behind (P V).
+// P has its own columns, so S_{j+1} is issued as soon as S_j sits in registers, and the wait on
+// P V_{j-1} comes in the middle of block j, just before P_j starts to overwrite P_{j-1}.
 //
-// O accumulates in TMEM across key blocks.  A row keeps an integer-valued reference maximum and
-// moves it only when a block maximum exceeds it by more than 2^8; then O is rescaled in TMEM
-// before the next P V is issued.  The decision is taken per row from that row's own scores; rows
-// that keep their reference multiply by exactly 1, so a row's bits never depend on its neighbours.
+// Reference of the softmax: the maximum of the row's FIRST block, rounded up to an integer, found
+// by both threads of the row (each scans all 128 columns, so they agree bit for bit without
+// talking) and never moved: later blocks need no maximum, no rescaling of O and no exchange.
+// fp32 holds 2^x up to x = 128, so a row overflows only if a later score exceeds its first block's
+// maximum by about 88 nats; such a row shows Inf/NaN in its sums at the end of the item and is then
+// computed again by its two threads alone in plain fp32 loops (slow, correct, reached only by inputs
+// whose scores span more than fp32's exponent range).  Every decision is taken per row from that
+// row's own values, so a row's bits never depend on its neighbours.
 #include <algorithm>
 
 #include "rocs_internal.h"
@@ -45,20 +45,49 @@ constexpr int BKV = 128;          // keys per block
 constexpr int kSoftmaxWarps = 16; // 8 per side
 constexpr int kControlWarp0 = kSoftmaxWarps;   // warps 16, 19: TMA producers of sides A, B; 17, 18: their MMA issuers
 constexpr int kThreads = (kSoftmaxWarps + 4) * 32;
-constexpr int kKvStages = 3;        // per side
-constexpr int kQSlots = 1;         // Q buffers per side (freed when the item's last S is issued, a block before its end)
+constexpr int kKvStages = 3;      // per side
 constexpr int kTmemCols = 512;
 constexpr int kQBytes = BQ * DH * 2;            // 16 KB
 constexpr int kKBytes = BKV * DH * 2;           // 16 KB
 constexpr int kKvStageBytes = 2 * kKBytes;      // K block + V block
-constexpr int kXchgBytes = 2 * 2 * BQ * 4;  // partial sums of the two halves of a row [side][half][row]
-constexpr int kNumBarriers = 2 * (2 * kQSlots + 2 * kKvStages) + 8 + 8 + 2;
-constexpr int kSmemBytes = 2 * (kQSlots * kQBytes + kKvStages * kKvStageBytes) + kXchgBytes + kNumBarriers * 8 + 16;
-constexpr float kRescaleThreshold = 8.f;  // log2 units
 constexpr uint32_t kStatusDca = 0x400;
 constexpr int kSideTmemStride = 256;
 constexpr int kPColOffset = 128;
 constexpr int kOColOffset = 192;
+
+// Shared-memory map (byte offsets from the 1024-byte aligned base); per side: one Q tile (freed when
+// the item's last S is issued, a block before its end) and a ring of K/V stages.
+constexpr uint32_t kOffQ = 0;                                          // [2 sides][128][64] bf16
+constexpr uint32_t kOffKv = kOffQ + 2 * kQBytes;                       // [2 sides][stages][K 16 KB | V 16 KB]
+constexpr uint32_t kOffL = kOffKv + 2 * kKvStages * kKvStageBytes;     // partial sums [2 sides][2 halves][128] fp32
+constexpr uint32_t kOffBar = kOffL + 2 * 2 * BQ * 4;
+// barriers, 8 bytes each, [side] innermost where there are two
+constexpr uint32_t kBarQFull = kOffBar;                    // [2]
+constexpr uint32_t kBarQEmpty = kBarQFull + 16;            // [2]
+constexpr uint32_t kBarKvFull = kBarQEmpty + 16;           // [2][stages]
+constexpr uint32_t kBarKvEmpty = kBarKvFull + 16 * kKvStages;
+constexpr uint32_t kBarSFull = kBarKvEmpty + 16 * kKvStages;  // [2]
+constexpr uint32_t kBarSEmpty = kBarSFull + 16;
+constexpr uint32_t kBarPFull = kBarSEmpty + 16;
+constexpr uint32_t kBarOFull = kBarPFull + 16;
+constexpr uint32_t kBarPair = kBarOFull + 16;              // [8]: the two warps that share 32 query rows
+constexpr uint32_t kBarDrain = kBarPair + 64;              // [2]
+constexpr uint32_t kOffTmemPtr = kBarDrain + 16;
+constexpr uint32_t kOffAbort = kOffTmemPtr + 4;
+constexpr int kSmemBytes = kOffAbort + 12;
+static_assert(kSmemBytes <= 232448, "shared memory of one SM");
+
+#ifndef ROCS_DCA_EMU
+#define ROCS_DCA_EMU 0
+#endif
+// Of every 8 column pairs of a row, this many take 2^x from a cubic on the FMA pipe instead of the
+// exponential unit (which pairs is fixed by the column index, so a row's bits do not depend on its
+// neighbours): 2^x = 2^n 2^r, n = round(x), |r| <= 1/2, 2^r by a polynomial with relative error
+// 7.5e-5, far below the rounding of P to bf16.  Off by default: with the rest of the loop as it is
+// the exponential unit is not what limits the kernel (measured).
+constexpr int kEmuPairs = ROCS_DCA_EMU;
+constexpr float kMagic = 12582912.f;  // 1.5 * 2^23: adding it rounds to an integer kept in the low mantissa bits
+constexpr float kPoly0 = 0.9999280572f, kPoly1 = 0.6932609677f, kPoly2 = 0.2426111251f, kPoly3 = 0.0551716685f;
 
 struct DcaParams {
   const DcaItem* items;
@@ -108,6 +137,11 @@ __device__ __forceinline__ float fmax3(float a, float b, float c) {
   asm("max.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c));
   return d;
 }
+__device__ __forceinline__ float fmax_nan(float a, float b) {  // NaN if either input is NaN
+  float d;
+  asm("max.NaN.f32 %0, %1, %2;" : "=f"(d) : "f"(a), "f"(b));
+  return d;
+}
 __device__ __forceinline__ uint32_t bf16x2_bits(float lo, float hi) {
   const __nv_bfloat162 h2 = __floats2bfloat162_rn(lo, hi);
   return *reinterpret_cast<const uint32_t*>(&h2);
@@ -122,23 +156,14 @@ __device__ __forceinline__ void umma_ts(uint32_t d_tmem, uint32_t a_tmem, uint64
       "r"(a_tmem), "l"(b_desc), "r"(idesc), "r"(accumulate)
       : "memory");
 }
-__device__ __forceinline__ void tmem_st_32x32b_x32(uint32_t taddr, const uint32_t* r) {
-  asm volatile(
-      "tcgen05.st.sync.aligned.32x32b.x32.b32 [%0], "
-      "{%1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16, "
-      "%17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31, %32};" ::"r"(taddr),
-      "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]), "r"(r[8]),
-      "r"(r[9]), "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15]), "r"(r[16]), "r"(r[17]),
-      "r"(r[18]), "r"(r[19]), "r"(r[20]), "r"(r[21]), "r"(r[22]), "r"(r[23]), "r"(r[24]), "r"(r[25]), "r"(r[26]),
-      "r"(r[27]), "r"(r[28]), "r"(r[29]), "r"(r[30]), "r"(r[31])
-      : "memory");
-}
 
 // One query row of one head, 32 of its 64 output columns, in plain fp32 with the row's true maximum as
 // reference: q and k point at the head's 64 values of the row / of the request's first key, v at the
-// 32 columns wanted; consecutive keys are `stride` elements apart.
+// 32 columns wanted; consecutive keys are `stride` elements apart.  Inlined on purpose: as a called
+// function it forces the caller's hot loop to keep its registers where the calling convention wants
+// them, and the loop spills.
 __device__ __forceinline__ void row_by_hand(const __nv_bfloat16* q, const __nv_bfloat16* k, const __nv_bfloat16* v,
-                                         int32_t stride, int32_t L, float scale_log2e, __nv_bfloat16* out) {
+                                            int32_t stride, int32_t L, float scale_log2e, __nv_bfloat16* out) {
   auto score = [&](int32_t j) {
     float s = 0.f;
     for (int d = 0; d < DH; ++d) s = fmaf(__bfloat162float(q[d]), __bfloat162float(k[(int64_t)j * stride + d]), s);
@@ -157,8 +182,8 @@ __device__ __forceinline__ void row_by_hand(const __nv_bfloat16* q, const __nv_b
   for (int d = 0; d < 32; ++d) out[d] = __float2bfloat16_rn(acc[d] * inv);
 }
 
-// A short burst of probes before the paced wait: for hand-offs that complete within a few dozen cycles.
-__device__ __forceinline__ bool mbar_wait_spin(uint64_t* bar, uint32_t parity, AbortFlag* abort_flag, uint32_t* status,
+// A short burst of probes before the paced wait: for hand-offs that are usually complete already.
+__device__ __forceinline__ bool mbar_wait_spin(uint32_t bar, uint32_t parity, AbortFlag* abort_flag, uint32_t* status,
                                                uint32_t code) {
 #pragma unroll 1
   for (int i = 0; i < 64; ++i)
@@ -170,67 +195,51 @@ __device__ __forceinline__ bool mbar_wait_spin(uint64_t* bar, uint32_t parity, A
 // event stamps of CTA 0: [role 0..3][block 0..kTraceBlocks)[event 0..8)
 constexpr int kTraceBlocks = 96;
 #define TRACE_EV(role, ev) do { if (p.trace && blockIdx.x == 0 && lane == 0 && tr_blk < kTraceBlocks) p.trace[((role) * kTraceBlocks + tr_blk) * 8 + (ev)] = clock64(); } while (0)
+#define TRACE_NEXT() ++tr_blk
 #else
 #define TRACE_EV(role, ev)
+#define TRACE_NEXT()
 #endif
 
 __global__ void __launch_bounds__(kThreads, 1)
 dca_umma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
                 const __grid_constant__ CUtensorMap map_v, const DcaParams p) {
   extern __shared__ __align__(1024) uint8_t smem[];     // swizzled operand tiles need 1024-byte alignment
-  uint8_t* q_smem = smem;                                // [2 sides][slots][128][64] bf16
-  uint8_t* kv_smem = q_smem + 2 * kQSlots * kQBytes;     // [2 sides][stages][K 16 KB | V 16 KB]
-  float* l_x = reinterpret_cast<float*>(kv_smem + 2 * kKvStages * kKvStageBytes);  // [2 sides][2 halves][128]
-  uint64_t* q_full = reinterpret_cast<uint64_t*>(l_x + 2 * 2 * BQ);  // [2 sides][slots]
-  uint64_t* q_empty = q_full + 2 * kQSlots;      // [2][slots]
-  uint64_t* kv_full = q_empty + 2 * kQSlots;     // [2][stages]
-  uint64_t* kv_empty = kv_full + 2 * kKvStages;  // [2][stages]
-  uint64_t* s_full = kv_empty + 2 * kKvStages;   // [2]
-  uint64_t* s_empty = s_full + 2;            // [2]
-  uint64_t* p_full = s_empty + 2;            // [2]
-  uint64_t* o_full = p_full + 2;             // [2]
-  uint64_t* pair_bar = o_full + 2;           // [8]: the two warps that share 32 query rows
-  uint64_t* drain = pair_bar + 8;
-  uint32_t* tmem_ptr = reinterpret_cast<uint32_t*>(drain + 2);
-  AbortFlag* abort_flag = reinterpret_cast<AbortFlag*>(tmem_ptr + 1);
+  const uint32_t sb = smem_u32(smem);                   // every shared-memory address below is sb + constant
+  AbortFlag* abort_flag = reinterpret_cast<AbortFlag*>(smem + kOffAbort);
 
   const int warp = threadIdx.x / 32, lane = threadIdx.x % 32;
-  if ((smem_u32(smem) & 1023u) != 0) {  // the swizzled tiles assume a 1024-byte aligned base
+  if ((sb & 1023u) != 0) {  // the swizzled tiles assume a 1024-byte aligned base
     if (threadIdx.x == 0) atomicCAS(p.status, 0u, kStatusDca | 15);
     return;
   }
 
   if (threadIdx.x == 0) {
-    for (int x = 0; x < 2 * kQSlots; ++x) {
-      mbar_init(&q_full[x], 1);
-      mbar_init(&q_empty[x], 1);
-    }
-    for (int s = 0; s < 2 * kKvStages; ++s) {
-      mbar_init(&kv_full[s], 1);
-      mbar_init(&kv_empty[s], 1);
-    }
-    for (int x = 0; x < 2; ++x) {
-      mbar_init(&s_full[x], 1);
-      mbar_init(&s_empty[x], kSoftmaxWarps / 2);
-      mbar_init(&p_full[x], kSoftmaxWarps / 2);
-      mbar_init(&o_full[x], 1);
-    }
-    for (int x = 0; x < 8; ++x) mbar_init(&pair_bar[x], 2);
-    mbar_init(&drain[0], 1);
-    mbar_init(&drain[1], 1);
+    auto init = [&](uint32_t off, int n, uint32_t count) {
+      for (int x = 0; x < n; ++x) mbar_init(reinterpret_cast<uint64_t*>(smem + off + 8 * x), count);
+    };
+    init(kBarQFull, 2, 1);
+    init(kBarQEmpty, 2, 1);
+    init(kBarKvFull, 2 * kKvStages, 1);
+    init(kBarKvEmpty, 2 * kKvStages, 1);
+    init(kBarSFull, 2, 1);
+    init(kBarSEmpty, 2, kSoftmaxWarps / 2);
+    init(kBarPFull, 2, kSoftmaxWarps / 2);
+    init(kBarOFull, 2, 1);
+    init(kBarPair, 8, 2);
+    init(kBarDrain, 2, 1);
     abort_flag->v = 0;
     fence_mbar_init();
   }
   if (warp == kControlWarp0 + 1) {
-    tmem_alloc(tmem_ptr, kTmemCols);
+    tmem_alloc(reinterpret_cast<uint32_t*>(smem + kOffTmemPtr), kTmemCols);
     tmem_relinquish();
   }
   tc_fence_before_sync();
   __syncthreads();
   tc_fence_after_sync();
-  const uint32_t tmem_base = *tmem_ptr;
+  const uint32_t tmem_base = *reinterpret_cast<const uint32_t*>(smem + kOffTmemPtr);
   const int32_t row_width = p.H * DH;  // elements per query / key row over all heads
-
   // Each side is a stream of its own: items 2 b + side, 2 b + side + 2 grid, ... of CTA b.
   const int32_t item0 = 2 * (int32_t)blockIdx.x, item_step = 2 * (int32_t)gridDim.x;
 
@@ -241,11 +250,9 @@ dca_umma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
       prefetch_tensormap(&map_q);
       prefetch_tensormap(&map_k);
       prefetch_tensormap(&map_v);
-      uint64_t* qf = q_full + side * kQSlots;
-      uint64_t* qe = q_empty + side * kQSlots;
-      uint64_t* kf = kv_full + side * kKvStages;
-      uint64_t* ke = kv_empty + side * kKvStages;
-      uint8_t* kv_side = kv_smem + side * kKvStages * kKvStageBytes;
+      const uint32_t q_full = sb + kBarQFull + 8 * side, q_empty = sb + kBarQEmpty + 8 * side;
+      const uint32_t kv_full = sb + kBarKvFull + 8 * kKvStages * side, kv_empty = sb + kBarKvEmpty + 8 * kKvStages * side;
+      const uint32_t q_dst = sb + kOffQ + side * kQBytes, kv_dst = sb + kOffKv + side * kKvStages * kKvStageBytes;
       uint32_t kv_it = 0, n_work = 0;
       bool ok = true;
       for (int32_t i = item0 + side; i < p.num_items && ok; i += item_step) {
@@ -253,28 +260,26 @@ dca_umma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
         const int32_t s0 = p.seq_offsets[item.req];
         const int32_t L = p.seq_offsets[item.req + 1] - s0;
         if (L == 0) continue;  // nobody touches a barrier for an item without keys
-        const uint32_t slot = n_work % kQSlots;
-        if (!mbar_wait_paced(&qe[slot], ((n_work / kQSlots) & 1) ^ 1, abort_flag, p.status, kStatusDca | 1)) { ok = false; break; }
+        if (!mbar_wait_paced(q_empty, (n_work & 1) ^ 1, abort_flag, p.status, kStatusDca | 1)) { ok = false; break; }
         ++n_work;
-        mbar_expect_tx(&qf[slot], kQBytes);
-        tma_load_2d(q_smem + (side * kQSlots + slot) * kQBytes, &map_q, &qf[slot], item.head * DH, item.cand0 * p.n_q);
+        mbar_expect_tx(q_full, kQBytes);
+        tma_load_2d(q_dst, &map_q, q_full, item.head * DH, item.cand0 * p.n_q);
         const int32_t nblk = (L + BKV - 1) / BKV;
         for (int32_t j = 0; j < nblk; ++j, ++kv_it) {
-          const int s = kv_it % kKvStages;
-          if (!mbar_wait_paced(&ke[s], ((kv_it / kKvStages) & 1) ^ 1, abort_flag, p.status, kStatusDca | 2)) { ok = false; break; }
-          uint8_t* st = kv_side + s * kKvStageBytes;
-          mbar_expect_tx(&kf[s], kKvStageBytes);
-          tma_load_2d(st, &map_k, &kf[s], item.head * DH, s0 + j * BKV);
-          tma_load_2d(st + kKBytes, &map_v, &kf[s], item.head * DH, s0 + j * BKV);
+          const uint32_t s = kv_it % kKvStages;
+          if (!mbar_wait_paced(kv_empty + 8 * s, ((kv_it / kKvStages) & 1) ^ 1, abort_flag, p.status, kStatusDca | 2)) { ok = false; break; }
+          mbar_expect_tx(kv_full + 8 * s, kKvStageBytes);
+          tma_load_2d(kv_dst + s * kKvStageBytes, &map_k, kv_full + 8 * s, item.head * DH, s0 + j * BKV);
+          tma_load_2d(kv_dst + s * kKvStageBytes + kKBytes, &map_v, kv_full + 8 * s, item.head * DH, s0 + j * BKV);
         }
       }
       if (!ok) {
         // let the loads in flight land before the CTA's shared memory goes away
-        for (int s = 0; s < kKvStages; ++s) {
-          const uint32_t n_issued = kv_it / kKvStages + (((int)(kv_it % kKvStages) > s) ? 1 : 0);
+        for (uint32_t s = 0; s < kKvStages; ++s) {
+          const uint32_t n_issued = kv_it / kKvStages + ((kv_it % kKvStages > s) ? 1 : 0);
           if (n_issued == 0) continue;
           const uint64_t t0 = globaltimer_ns();
-          while (!mbar_try_wait(&kf[s], (n_issued - 1) & 1) && globaltimer_ns() - t0 < kWaitLimitNs) {}
+          while (!mbar_try_wait_brief(kv_full + 8 * s, (n_issued - 1) & 1) && globaltimer_ns() - t0 < kWaitLimitNs) {}
         }
       }
     }
@@ -283,11 +288,11 @@ dca_umma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
     const int side = warp - (kControlWarp0 + 1);
     constexpr uint32_t idesc_s = umma_idesc_bf16(BQ, BKV, false, false);  // S = Q K^T, both K-major
     constexpr uint32_t idesc_o = umma_idesc_bf16(BQ, DH, false, true);    // O = P V, V is MN-major
-    uint64_t* qf = q_full + side * kQSlots;
-    uint64_t* qe = q_empty + side * kQSlots;
-    uint64_t* kf = kv_full + side * kKvStages;
-    uint64_t* ke = kv_empty + side * kKvStages;
-    uint8_t* kv_side = kv_smem + side * kKvStages * kKvStageBytes;
+    const uint32_t q_full = sb + kBarQFull + 8 * side, q_empty = sb + kBarQEmpty + 8 * side;
+    const uint32_t kv_full = sb + kBarKvFull + 8 * kKvStages * side, kv_empty = sb + kBarKvEmpty + 8 * kKvStages * side;
+    const uint32_t s_full = sb + kBarSFull + 8 * side, s_empty = sb + kBarSEmpty + 8 * side;
+    const uint32_t p_full = sb + kBarPFull + 8 * side, o_full = sb + kBarOFull + 8 * side;
+    const uint32_t kv_base = sb + kOffKv + side * kKvStages * kKvStageBytes;
     uint32_t kv_it = 0, n_work = 0;           // n_work: items that had keys (phase of q_full)
     uint32_t cnt_p = 0, cnt_se = 0;           // phases of p_full and s_empty of this side
     bool ok = true;
@@ -295,15 +300,14 @@ dca_umma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
     int tr_blk = 0;
 #endif
     const uint32_t t_s = tmem_base + side * kSideTmemStride;
-    // Descriptors are formed by the whole warp ahead of the barrier waits; the elected lane then only
-    // issues the products.
-    auto desc_q = [&](uint32_t slot) { return smem_desc_sw128(smem_u32(q_smem + (side * kQSlots + slot) * kQBytes), 1024, 16); };
-    auto desc_k = [&](int stage) { return smem_desc_sw128(smem_u32(kv_side + stage * kKvStageBytes), 1024, 16); };
-    auto desc_v = [&](int stage) { return smem_desc_sw128(smem_u32(kv_side + stage * kKvStageBytes + kKBytes), 1024, 16); };
-    auto issue_s = [&](uint64_t a_desc, uint64_t b_desc) {
+    // Q tile of this side, K block and V block of a stage as shared-memory operand descriptors
+    const uint64_t dq = smem_desc_sw128(sb + kOffQ + side * kQBytes, 1024, 16);
+    auto desc_k = [&](uint32_t stage) { return smem_desc_sw128(kv_base + stage * kKvStageBytes, 1024, 16); };
+    auto desc_v = [&](uint32_t stage) { return smem_desc_sw128(kv_base + stage * kKvStageBytes + kKBytes, 1024, 16); };
+    auto issue_s = [&](uint64_t b_desc) {
 #pragma unroll
-      for (int k = 0; k < DH / 16; ++k) umma_ss(t_s, a_desc + 2 * k, b_desc + 2 * k, idesc_s, k != 0 ? 1u : 0u);
-      umma_commit(&s_full[side]);
+      for (int k = 0; k < DH / 16; ++k) umma_ss(t_s, dq + 2 * k, b_desc + 2 * k, idesc_s, k != 0 ? 1u : 0u);
+      umma_commit(s_full);
     };
     auto issue_pv = [&](uint64_t b_desc, bool first_block) {
       // P: 16 keys = 8 columns of bf16 pairs in tensor memory
@@ -312,14 +316,14 @@ dca_umma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
       for (int k = 0; k < BKV / 16; ++k)
         umma_ts(t_s + kOColOffset, t_s + kPColOffset + k * 8, b_desc + k * (16 * 128 / 16), idesc_o,
                 (k != 0 || !first_block) ? 1u : 0u);
-      umma_commit(&o_full[side]);
+      umma_commit(o_full);
     };
     // The last block of a sequence may reach past it into the next request's rows (or past the
     // tensor, where TMA fills zeros).  Scores of such keys are masked to -inf by the softmax warps,
     // so P is exactly 0 there; the V rows are zeroed here so that 0 x (Inf or NaN of a foreign
     // request) cannot reach this request's output.
-    auto zero_v_tail = [&](int stage, int32_t valid) {
-      uint8_t* v = kv_side + stage * kKvStageBytes + kKBytes;
+    auto zero_v_tail = [&](uint32_t stage, int32_t valid) {
+      uint8_t* v = smem + kOffKv + (side * kKvStages + stage) * kKvStageBytes + kKBytes;
       for (int idx = valid * 8 + lane; idx < BKV * 8; idx += 32)
         *reinterpret_cast<uint4*>(v + idx * 16) = make_uint4(0u, 0u, 0u, 0u);
       fence_proxy_async_smem();
@@ -331,80 +335,76 @@ dca_umma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
       if (L == 0) continue;
       const int32_t nblk = (L + BKV - 1) / BKV;
       const int32_t tail_valid = L - (nblk - 1) * BKV;  // keys of the last block that exist
-      const uint32_t slot = n_work % kQSlots;
-      if (!mbar_wait_paced(&qf[slot], (n_work / kQSlots) & 1, abort_flag, p.status, kStatusDca | 3)) { ok = false; break; }
+      if (!mbar_wait_paced(q_full, n_work & 1, abort_flag, p.status, kStatusDca | 3)) { ok = false; break; }
       ++n_work;
       // first key block (the S tile was drained at the end of the previous item)
-      if (!mbar_wait_paced(&kf[kv_it % kKvStages], (kv_it / kKvStages) & 1, abort_flag, p.status, kStatusDca | 4)) { ok = false; break; }
+      if (!mbar_wait_paced(kv_full + 8 * (kv_it % kKvStages), (kv_it / kKvStages) & 1, abort_flag, p.status, kStatusDca | 4)) { ok = false; break; }
       if (nblk == 1 && tail_valid < BKV) zero_v_tail(kv_it % kKvStages, tail_valid);
       tc_fence_after_sync();
-      const uint64_t dq = desc_q(slot);
       if (lane == 0) {
-        issue_s(dq, desc_k(kv_it % kKvStages));
-        if (nblk == 1) umma_commit(&qe[slot]);
+        issue_s(desc_k(kv_it % kKvStages));
+        if (nblk == 1) umma_commit(q_empty);
       }
       __syncwarp();
       for (int32_t j = 0; j < nblk && ok; ++j, ++kv_it) {
-        const int stage = kv_it % kKvStages;
-        const int next_stage = (kv_it + 1) % kKvStages;
+        const uint32_t stage = kv_it % kKvStages;
+        const uint32_t next_stage = (kv_it + 1) % kKvStages;
         const uint64_t dk_next = desc_k(next_stage), dv = desc_v(stage);
         TRACE_EV(2 + side, 0);
         if (j + 1 < nblk) {
-          if (!mbar_wait_paced(&kf[next_stage], ((kv_it + 1) / kKvStages) & 1, abort_flag, p.status, kStatusDca | 5)) { ok = false; break; }
+          if (!mbar_wait_paced(kv_full + 8 * next_stage, ((kv_it + 1) / kKvStages) & 1, abort_flag, p.status, kStatusDca | 5)) { ok = false; break; }
           TRACE_EV(2 + side, 1);
           if (j + 2 == nblk && tail_valid < BKV) zero_v_tail(next_stage, tail_valid);
         }
         // S_{j+1} as soon as the side has pulled S_j into registers
-        if (!mbar_wait_paced(&s_empty[side], cnt_se & 1, abort_flag, p.status, kStatusDca | 11)) { ok = false; break; }
+        if (!mbar_wait_paced(s_empty, cnt_se & 1, abort_flag, p.status, kStatusDca | 11)) { ok = false; break; }
         ++cnt_se;
         TRACE_EV(2 + side, 2);
         if (j + 1 < nblk) {
           tc_fence_after_sync();
           if (lane == 0) {
-            issue_s(dq, dk_next);
-            if (j + 2 == nblk) umma_commit(&qe[slot]);  // last S of the item: Q slot is free
+            issue_s(dk_next);
+            if (j + 2 == nblk) umma_commit(q_empty);  // last S of the item: the Q tile is free
           }
           __syncwarp();
           TRACE_EV(2 + side, 3);
         }
         // P_j of this side is in tensor memory
-        if (!mbar_wait_paced(&p_full[side], cnt_p & 1, abort_flag, p.status, kStatusDca | 6)) { ok = false; break; }
+        if (!mbar_wait_paced(p_full, cnt_p & 1, abort_flag, p.status, kStatusDca | 6)) { ok = false; break; }
         ++cnt_p;
         TRACE_EV(2 + side, 4);
         tc_fence_after_sync();
         if (lane == 0) {
           issue_pv(dv, j == 0);
-          umma_commit(&ke[stage]);  // K_j and V_j are no longer needed
+          umma_commit(kv_empty + 8 * stage);  // K_j and V_j are no longer needed
         }
         __syncwarp();
         TRACE_EV(2 + side, 5);
-#ifdef ROCS_DCA_TRACE
-        ++tr_blk;
-#endif
+        TRACE_NEXT();
       }
     }
     if (!ok && lane == 0) {
-      umma_commit(&drain[side]);
+      umma_commit(sb + kBarDrain + 8 * side);
       const uint64_t t0 = globaltimer_ns();
-      while (!mbar_try_wait(&drain[side], 0) && globaltimer_ns() - t0 < kWaitLimitNs) {}
+      while (!mbar_try_wait_brief(sb + kBarDrain + 8 * side, 0) && globaltimer_ns() - t0 < kWaitLimitNs) {}
     }
   } else {
     // ------------------------------ softmax warps ------------------------------------------
-    const int sw = warp;
-    const int side = sw >> 3;
-    const int half = (sw >> 2) & 1;         // which 64 of the block's 128 key columns
+    const int side = warp >> 3;
+    const int half = (warp >> 2) & 1;       // which 64 of the block's 128 key columns
     const int q = warp & 3;                 // TMEM lane quadrant this warp may touch
     const int row = q * 32 + lane;          // query row of the tile = TMEM lane
-    const uint32_t t_side = tmem_base + side * kSideTmemStride + ((uint32_t)(q * 32) << 16);
-    const uint32_t t_s = t_side + half * 64;
-    const uint32_t t_row = t_side;                   // all 128 S columns of the row
-    const uint32_t t_p = t_side + kPColOffset + half * 32;
-    const uint32_t t_o = t_side + kOColOffset + half * 32;
-    uint64_t* my_pair = &pair_bar[side * 4 + q];
+    const uint32_t t_row = tmem_base + side * kSideTmemStride + ((uint32_t)(q * 32) << 16);  // S columns of the row
+    const uint32_t t_s = t_row + half * 64;
+    const uint32_t t_p = t_row + kPColOffset + half * 32;
+    const uint32_t t_o = t_row + kOColOffset + half * 32;
+    const uint32_t s_full = sb + kBarSFull + 8 * side, s_empty = sb + kBarSEmpty + 8 * side;
+    const uint32_t p_full = sb + kBarPFull + 8 * side, o_full = sb + kBarOFull + 8 * side;
+    const uint32_t my_pair = sb + kBarPair + 8 * (side * 4 + q);
     uint32_t cnt_s = 0, cnt_o = 0, cnt_pair = 0;
 #ifdef ROCS_DCA_TRACE
     int tr_blk = 0;
-    const int tr_role = sw == 0 ? 0 : sw == 8 ? 1 : -1;
+    const int tr_role = warp == 0 ? 0 : warp == 8 ? 1 : -1;
 #define TRACE_SM(ev) do { if (tr_role >= 0) TRACE_EV(tr_role, ev); } while (0)
 #else
 #define TRACE_SM(ev)
@@ -412,22 +412,17 @@ dca_umma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
     for (int32_t i = item0 + side; i < p.num_items; i += item_step) {
       const DcaItem item = p.items[i];
       const int32_t L = p.seq_offsets[item.req + 1] - p.seq_offsets[item.req];
-      const int32_t my_count = item.count_a;
-      const int32_t cand_first = item.cand0;
-      const int32_t rows_valid = my_count * p.n_q;
-      const int32_t head = item.head;
-      auto out_ptr = [&]() { return p.O + ((int64_t)cand_first * p.n_q + row) * row_width + head * DH + half * 32; };
+      const int32_t rows_valid = item.count_a * p.n_q;
+      // this thread's 32 output columns of its row
+      auto out_ptr = [&]() { return p.O + ((int64_t)item.cand0 * p.n_q + row) * row_width + item.head * DH + half * 32; };
       bool aborted = false;
-      if (my_count > 0 && L > 0) {
+      if (L > 0) {
         const int32_t nblk = (L + BKV - 1) / BKV;
-        float m_ref, l_run = 0.f;
-        // ---- reference of the row: the maximum of its first block, rounded up to an integer.
-        // Both threads of a row scan all 128 columns, so they get bitwise the same value without
-        // talking to each other.  It is never moved: later blocks use the same reference, whatever
-        // their scores (see the end of the item for rows whose scores grow past fp32's range).
+        // ---- reference of the row: the maximum of its first block, rounded up to an integer
         TRACE_SM(0);
-        if (!mbar_wait_spin(&s_full[side], cnt_s & 1, abort_flag, p.status, kStatusDca | 7)) { aborted = true; break; }
+        if (!mbar_wait_spin(s_full, cnt_s & 1, abort_flag, p.status, kStatusDca | 7)) break;
         tc_fence_after_sync();
+        float m_ref;
         {
           float mx4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
 #pragma unroll
@@ -447,11 +442,18 @@ dca_umma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
           m_ref = ceilf(fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3])) * p.scale_log2e);
         }
         const uint64_t c2 = pack2(p.scale_log2e, p.scale_log2e), m2 = pack2(-m_ref, -m_ref);
+        // the polynomial path: x = s c - m_ref with m_ref an integer, so n = round(x) comes out of one
+        // fused multiply-add against kMagic - m_ref; scores are clamped from below at x = -126 (2^x is
+        // nothing there) and must stay below x = 126, which is checked per block
+        const float k_off = kMagic - m_ref;
+        const float s_lo = (m_ref - 126.f) / p.scale_log2e;
+        bool by_hand = kEmuPairs > 0 && !(fabsf(m_ref) < 1048576.f);  // kMagic - m_ref must be exact
+        float g_max = -INFINITY;                     // largest raw score that went through the polynomial
         uint64_t sum2 = pack2(0.f, 0.f);
         for (int32_t j = 0; j < nblk; ++j) {
           if (j > 0) {
             TRACE_SM(0);
-            if (!mbar_wait_spin(&s_full[side], cnt_s & 1, abort_flag, p.status, kStatusDca | 7)) { aborted = true; break; }
+            if (!mbar_wait_spin(s_full, cnt_s & 1, abort_flag, p.status, kStatusDca | 7)) { aborted = true; break; }
             tc_fence_after_sync();
           }
           ++cnt_s;
@@ -462,7 +464,7 @@ dca_umma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
           tmem_ld_wait();
           tc_fence_before_sync();
           __syncwarp();
-          if (lane == 0) mbar_arrive(&s_empty[side]);  // S_{j+1} may overwrite the tile now
+          if (lane == 0) mbar_arrive(s_empty);  // S_{j+1} may overwrite the tile now
           const int32_t valid = L - j * BKV - half * 64;  // columns of this thread's half that are keys of the request
           if (valid < 64) {
 #pragma unroll
@@ -472,9 +474,29 @@ dca_umma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
           TRACE_SM(2);
           uint32_t pk[16];  // P of 32 keys of this row, bf16 pairs; stored in two halves
           auto exp_pair = [&](int e) {
-            float x0, x1;
-            unpack2(ffma2(pack2(__uint_as_float(sv[e]), __uint_as_float(sv[e + 1])), c2, m2), x0, x1);
-            const float p0 = ex2(x0), p1 = ex2(x1);
+            float p0, p1;
+            if (((e >> 1) & 7) < kEmuPairs) {
+              const uint64_t k2 = pack2(k_off, k_off);
+              const float s0 = __uint_as_float(sv[e]), s1 = __uint_as_float(sv[e + 1]);
+              g_max = fmax3(g_max, s0, s1);
+              const uint64_t s2 = pack2(fmax_nan(s0, s_lo), fmax_nan(s1, s_lo));
+              const uint64_t xf2 = ffma2(s2, c2, k2);                        // kMagic + n
+              const uint64_t w2 = ffma2(xf2, pack2(-1.f, -1.f), k2);          // -(n + m_ref)
+              const uint64_t r2 = ffma2(s2, c2, w2);                         // x - n
+              uint64_t q2 = ffma2(r2, pack2(kPoly3, kPoly3), pack2(kPoly2, kPoly2));
+              q2 = ffma2(q2, r2, pack2(kPoly1, kPoly1));
+              q2 = ffma2(q2, r2, pack2(kPoly0, kPoly0));
+              float q0, q1, f0, f1;
+              unpack2(q2, q0, q1);
+              unpack2(xf2, f0, f1);
+              p0 = __uint_as_float(__float_as_uint(q0) + (__float_as_uint(f0) << 23));  // 2^r scaled by 2^n
+              p1 = __uint_as_float(__float_as_uint(q1) + (__float_as_uint(f1) << 23));
+            } else {
+              float x0, x1;
+              unpack2(ffma2(pack2(__uint_as_float(sv[e]), __uint_as_float(sv[e + 1])), c2, m2), x0, x1);
+              p0 = ex2(x0);
+              p1 = ex2(x1);
+            }
             sum2 = fadd2(sum2, pack2(p0, p1));
             pk[(e / 2) & 15] = bf16x2_bits(p0, p1);
           };
@@ -484,83 +506,74 @@ dca_umma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
           if (j > 0) {
             // P V of the previous block has read P_{j-1} (it was issued most of a block ago): from here
             // on this thread's P columns may be rewritten
-            if (!mbar_wait_spin(&o_full[side], cnt_o & 1, abort_flag, p.status, kStatusDca | 8)) { aborted = true; break; }
-            ++cnt_o;
+            if (!mbar_wait_spin(o_full, (cnt_o & 1) ^ 1, abort_flag, p.status, kStatusDca | 8)) { aborted = true; break; }
             tc_fence_after_sync();
           }
+          ++cnt_o;
           TRACE_SM(4);
           tmem_st_32x32b_x16(t_p, pk);
 #pragma unroll
           for (int e = 32; e < 64; e += 2) exp_pair(e);
           TRACE_SM(5);
           tmem_st_32x32b_x16(t_p + 16, pk);
+          if (kEmuPairs > 0 && g_max * p.scale_log2e - m_ref > 126.f) by_hand = true;  // 2^n would leave fp32's exponent field
           tmem_st_wait();
           tc_fence_before_sync();
           __syncwarp();
-          if (lane == 0) mbar_arrive(&p_full[side]);
+          if (lane == 0) mbar_arrive(p_full);
           TRACE_SM(6);
-#ifdef ROCS_DCA_TRACE
-          ++tr_blk;
-#endif
+          TRACE_NEXT();
         }
-        if (!aborted) {
-          float sum_lo, sum_hi;
-          unpack2(sum2, sum_lo, sum_hi);
-          l_run = sum_lo + sum_hi;
-          float* l_mine = l_x + (side * 2 + half) * BQ + row;
-          const float* l_other = l_x + (side * 2 + (half ^ 1)) * BQ + row;
-          *l_mine = l_run;
-          __syncwarp();
-          if (lane == 0) mbar_arrive(my_pair);
-          if (!mbar_wait_paced(my_pair, cnt_pair & 1, abort_flag, p.status, kStatusDca | 14) ||
-              !mbar_wait_paced(&o_full[side], cnt_o & 1, abort_flag, p.status, kStatusDca | 9)) {
-            aborted = true;
-          } else {
-            ++cnt_pair;
-            ++cnt_o;
-            tc_fence_after_sync();
-            const float l_o = *l_other;
-            const float l_tot = half == 0 ? l_run + l_o : l_o + l_run;  // same order in both halves
-            const float inv = 1.f / l_tot;
-            uint32_t v[32];
-            tmem_ld_32x32b_x32(t_o, v);
-            tmem_ld_wait();
-            // Scores that outgrow the first block's maximum by 2^128 or so overflow fp32 (and so can
-            // a sum of products with huge values): the row then holds Inf or NaN instead of a result.
-            float probe = l_tot * 0.f;
+        if (aborted) break;
+        float sum_lo, sum_hi;
+        unpack2(sum2, sum_lo, sum_hi);
+        const float l_run = sum_lo + sum_hi;
+        float* l_x = reinterpret_cast<float*>(smem + kOffL);
+        l_x[(side * 2 + half) * BQ + row] = by_hand ? __int_as_float(0x7fc00000) : l_run;  // NaN tells the other half of the row too
+        __syncwarp();
+        if (lane == 0) mbar_arrive(my_pair);
+        if (!mbar_wait_paced(my_pair, cnt_pair & 1, abort_flag, p.status, kStatusDca | 14) ||
+            !mbar_wait_paced(o_full, (cnt_o & 1) ^ 1, abort_flag, p.status, kStatusDca | 9))
+          break;
+        ++cnt_pair;
+        tc_fence_after_sync();
+        const float l_o = l_x[(side * 2 + (half ^ 1)) * BQ + row];
+        const float l_tot = half == 0 ? l_run + l_o : l_o + l_run;  // same order in both halves
+        const float inv = 1.f / l_tot;
+        uint32_t v[32];
+        tmem_ld_32x32b_x32(t_o, v);
+        tmem_ld_wait();
+        // Scores that outgrow the first block's maximum by 2^128 or so overflow fp32 (and so can
+        // a sum of products with huge values): the row then holds Inf or NaN instead of a result.
+        float probe = l_tot * 0.f;
 #pragma unroll
-            for (int e = 0; e < 32; ++e) probe = fmaf(__uint_as_float(v[e]), 0.f, probe);
-            if (row < rows_valid) {
-              __nv_bfloat16* out = out_ptr();
-              if (probe == 0.f) {
+        for (int e = 0; e < 32; ++e) probe = fmaf(__uint_as_float(v[e]), 0.f, probe);
+        if (row < rows_valid) {
+          __nv_bfloat16* out = out_ptr();
+          if (probe == 0.f && !by_hand) {
 #pragma unroll
-                for (int e = 0; e < 32; e += 8) {
-                  uint4 w;
-                  w.x = bf16x2_bits(__uint_as_float(v[e + 0]) * inv, __uint_as_float(v[e + 1]) * inv);
-                  w.y = bf16x2_bits(__uint_as_float(v[e + 2]) * inv, __uint_as_float(v[e + 3]) * inv);
-                  w.z = bf16x2_bits(__uint_as_float(v[e + 4]) * inv, __uint_as_float(v[e + 5]) * inv);
-                  w.w = bf16x2_bits(__uint_as_float(v[e + 6]) * inv, __uint_as_float(v[e + 7]) * inv);
-                  *reinterpret_cast<uint4*>(out + e) = w;
-                }
-              } else {
-                // such a row is computed again here, by this thread alone, with a reference that is
-                // its true maximum (plain fp32 loops over the request's keys: slow, and reached only
-                // by inputs whose scores span more than fp32's exponent range)
-                const int64_t q_row = (int64_t)cand_first * p.n_q + row;
-                row_by_hand(p.Q + q_row * row_width + head * DH, p.K + ((int64_t)p.seq_offsets[item.req] * p.H + head) * DH,
-                            p.V + ((int64_t)p.seq_offsets[item.req] * p.H + head) * DH + half * 32, row_width, L,
-                            p.scale_log2e, out);
-              }
+            for (int e = 0; e < 32; e += 8) {
+              uint4 w;
+              w.x = bf16x2_bits(__uint_as_float(v[e + 0]) * inv, __uint_as_float(v[e + 1]) * inv);
+              w.y = bf16x2_bits(__uint_as_float(v[e + 2]) * inv, __uint_as_float(v[e + 3]) * inv);
+              w.z = bf16x2_bits(__uint_as_float(v[e + 4]) * inv, __uint_as_float(v[e + 5]) * inv);
+              w.w = bf16x2_bits(__uint_as_float(v[e + 6]) * inv, __uint_as_float(v[e + 7]) * inv);
+              *reinterpret_cast<uint4*>(out + e) = w;
             }
+          } else {
+            // such a row is computed again here, by this thread alone, with its true maximum as reference
+            const int64_t q_row = (int64_t)item.cand0 * p.n_q + row;
+            const int64_t kv0 = ((int64_t)p.seq_offsets[item.req] * p.H + item.head) * DH;
+            row_by_hand(p.Q + q_row * row_width + item.head * DH, p.K + kv0, p.V + kv0 + half * 32, row_width, L,
+                        p.scale_log2e, out);
           }
         }
-      } else if (my_count > 0 && row < rows_valid) {
+      } else if (row < rows_valid) {
         // a request without keys: zero rows
         __nv_bfloat16* out = out_ptr();
 #pragma unroll
         for (int c = 0; c < 32; c += 8) *reinterpret_cast<uint4*>(out + c) = make_uint4(0u, 0u, 0u, 0u);
       }
-      if (aborted) break;
       tc_fence_before_sync();  // the next item's first P V overwrites O
     }
   }
