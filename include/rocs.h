@@ -131,7 +131,12 @@ rocs_status_t rocs_ikbo_linear(const rocs_plan_t* plan, rocs_dtype_t dtype, int3
  *   cand_offsets [R+1] device int32 as for rocs_plan_create; its contents are not validated
  *   (they live on the device).  d_req, d_cand, d_out > 0.  Other arguments as above.
  *   The first call on a device looks up the array's device address (cudaGetSymbolAddress);
- *   make that first call outside any stream capture.
+ *   make that first call outside any stream capture.  The CUDA runtime itself loads a kernel's
+ *   code the first time that kernel is launched, which can allocate: which kernels run depends
+ *   on the shape class (dtype, small or large N, width of d_out), so a host with a frozen
+ *   allocator should send one warm-up call per shape class it will use at start-up (or run with
+ *   CUDA_MODULE_LOADING=EAGER).  rocs_set_path does not apply to this entry point: it always
+ *   takes the tensor-core kernels where the shape allows.
  *   All calls share the one array, and it keeps whatever the previous call left.  Each call
  *   overwrites every word it later reads, so stale contents are harmless, but two calls whose
  *   kernels overlap on the GPU (different streams, no ordering between them) race on it:

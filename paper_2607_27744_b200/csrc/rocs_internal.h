@@ -114,13 +114,8 @@ rocs_status_t umma_linear(int64_t M, int32_t d_in, int32_t d_out, const void* X,
                           const void* W, int64_t ld_w, const float* bias, const float* add,
                           int64_t ld_add, const int32_t* row2req, int act, void* Y, int64_t ld_y,
                           bool out_f32, cudaStream_t stream, bool add_from_previous_launch = false);
-// Weight-stationary variant for d_in <= 256 and bf16 output (umma_linear picks it when it applies).
-bool umma_linear_ws_supported(int64_t M, int32_t d_in, int32_t d_out, bool out_f32);
-rocs_status_t umma_linear_ws(int64_t M, int32_t d_in, int32_t d_out, const void* X, int64_t ld_x,
-                             const void* W, int64_t ld_w, const float* bias, const float* add,
-                             int64_t ld_add, const int32_t* row2req, int act, void* Y, int64_t ld_y,
-                             cudaStream_t stream);
-// The same on CTA pairs (cta_group::2): half a weight slice per SM, TMA-store epilogue.
+// Weight-stationary kernel on CTA pairs (cta_group::2) for d_in <= 256 and bf16 output: half a weight
+// slice per SM, TMA-store epilogue (umma_linear picks it when it applies).
 bool umma_linear_ws2_supported(int64_t M, int32_t d_in, int32_t d_out, bool out_f32);
 rocs_status_t umma_linear_ws2(int64_t M, int32_t d_in, int32_t d_out, const void* X, int64_t ld_x,
                               const void* W, int64_t ld_w, const float* bias, const float* add,

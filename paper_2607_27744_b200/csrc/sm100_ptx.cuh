@@ -58,7 +58,7 @@ struct AbortFlag {
 // Waits for the phase with the given parity.  Returns false if the CTA is aborting or the wait
 // expired (then `code` is recorded in *status and the abort flag is raised).
 __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, AbortFlag* abort_flag,
-                                          uint32_t* status, uint32_t code) {
+                                          uint32_t* status, uint32_t code, uint64_t limit_ns = kWaitLimitNs) {
   if (mbar_try_wait(bar, parity)) return true;
   const uint64_t t0 = globaltimer_ns();
   while (true) {
@@ -68,7 +68,7 @@ __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, AbortF
     for (int poll = 0; poll < 16; ++poll)
       if (mbar_try_wait(bar, parity)) return true;
     if (abort_flag->v) return false;
-    if (globaltimer_ns() - t0 > kWaitLimitNs) {
+    if (globaltimer_ns() - t0 > limit_ns) {
       abort_flag->v = 1;
       atomicCAS(status, 0u, code);
       return false;
@@ -91,13 +91,13 @@ __device__ __forceinline__ bool mbar_try_wait_brief(uint64_t* bar, uint32_t pari
   return ok != 0;
 }
 __device__ __forceinline__ bool mbar_wait_paced(uint64_t* bar, uint32_t parity, AbortFlag* abort_flag,
-                                                uint32_t* status, uint32_t code) {
+                                                uint32_t* status, uint32_t code, uint64_t limit_ns = kWaitLimitNs) {
   if (mbar_try_wait_brief(bar, parity)) return true;
   const uint64_t t0 = globaltimer_ns();
   while (true) {
     if (mbar_try_wait_brief(bar, parity)) return true;
     if (abort_flag->v) return false;
-    if (globaltimer_ns() - t0 > kWaitLimitNs) {
+    if (globaltimer_ns() - t0 > limit_ns) {
       abort_flag->v = 1;
       atomicCAS(status, 0u, code);
       return false;
@@ -265,13 +265,13 @@ __device__ __forceinline__ bool mbar_try_wait_brief(uint32_t bar, uint32_t parit
   return ok != 0;
 }
 __device__ __forceinline__ bool mbar_wait_paced(uint32_t bar, uint32_t parity, AbortFlag* abort_flag, uint32_t* status,
-                                                uint32_t code) {
+                                                uint32_t code, uint64_t limit_ns = kWaitLimitNs) {
   if (mbar_try_wait_brief(bar, parity)) return true;
   const uint64_t t0 = globaltimer_ns();
   while (true) {
     if (mbar_try_wait_brief(bar, parity)) return true;
     if (abort_flag->v) return false;
-    if (globaltimer_ns() - t0 > kWaitLimitNs) {
+    if (globaltimer_ns() - t0 > limit_ns) {
       abort_flag->v = 1;
       atomicCAS(status, 0u, code);
       return false;

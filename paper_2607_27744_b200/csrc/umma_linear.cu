@@ -320,8 +320,6 @@ rocs_status_t umma_linear(int64_t M, int32_t d_in, int32_t d_out, const void* X,
                            add_from_previous_launch);
   if (umma_linear_pair_supported(M, d_in, d_out, out_f32, add != nullptr))
     return umma_linear_pair(M, d_in, d_out, X, ld_x, W, ld_w, bias, act, Y, ld_y, stream);
-  if (umma_linear_ws_supported(M, d_in, d_out, out_f32))
-    return umma_linear_ws(M, d_in, d_out, X, ld_x, W, ld_w, bias, add, ld_add, row2req, act, Y, ld_y, stream);
 #define ROCS_LAUNCH(BN_)                                                                                   \
   (out_f32 ? launch<BN_, float>(M, d_in, d_out, X, ld_x, W, ld_w, bias, add, ld_add, row2req, act, Y, ld_y, \
                                 stream)                                                                    \

@@ -28,7 +28,7 @@ constexpr int kStageBytes = kABytes + kBBytes;
 constexpr int kStages = 6;
 constexpr int kStagingBytes = kEpiWarps * 4096;  // one 32-row x 128-byte box per warp, used by both column chunks
 constexpr int kSmemBytes = kStages * kStageBytes + kStagingBytes + 512 + 1024;
-constexpr uint32_t kStatusPair = 0x600;
+constexpr uint32_t kStatusPair = 0x300;
 
 struct PairParams {
   int64_t M;

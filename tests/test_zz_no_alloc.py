@@ -9,6 +9,7 @@ import numpy as np
 import pytest
 import torch
 
+from oracle import rocs_ref as ref
 from paper_2607_27744_b200 import binding as rocs, workloads as wl
 from _util import rel_err, to_dev, to_host_f64, tol_for
 
@@ -36,6 +37,38 @@ def test_static_entry_matches_regular_entry_on_two_calls_in_a_row(cfg_id, dtype)
         rocs.ikbo_linear_static(co_d, XR, XC, W_CR, W_CC, got, bias=bias, relu=True)
         torch.cuda.synchronize()
         assert rel_err(to_host_f64(got), to_host_f64(want)) <= tol_for(dtype)
+    rocs.last_device_status()
+
+
+def test_static_entry_on_the_batch_sizes_real_callers_send():
+    """Batches large enough for the tensor-core candidate kernel (request rows fetched by TMA from
+    the fixed array, segments that change inside 32-row slabs), two calls in a row with different
+    request counts; checked against the regular entry point AND the CPU oracle; after a warm-up
+    call the device's free memory must not move across a call."""
+    cfg = wl.CONFIGS[2].with_(d_req=256, d_cand=128, d_out=192)
+    first = True
+    for counts in ([700, 3, 41, 0, 520, 17, 300], [33, 1290, 5]):
+        c = cfg.with_(R=len(counts))
+        co = wl.offsets_from_counts(counts)
+        d = wl.linear_inputs(c, co, bias=True)
+        W = to_dev(d["W"])
+        co_d, XR, XC, bias = to_dev(co), to_dev(d["XR"]), to_dev(d["XC"]), to_dev(d["bias"])
+        W_CR, W_CC = W[:, :c.d_req], W[:, c.d_req:]
+        plan = rocs.plan_create(co_d, co)
+        want = rocs.ikbo_linear(plan, XR, XC, W_CR, W_CC, bias=bias, relu=True)
+        got = torch.full_like(want, float("nan"))
+        if first:  # warm-up: first use of the kernels loads their code
+            rocs.ikbo_linear_static(co_d, XR, XC, W_CR, W_CC, got, bias=bias, relu=True)
+            torch.cuda.synchronize()
+            got.fill_(float("nan"))
+            first = False
+        free_before = torch.cuda.mem_get_info()[0]
+        rocs.ikbo_linear_static(co_d, XR, XC, W_CR, W_CC, got, bias=bias, relu=True)
+        torch.cuda.synchronize()
+        assert torch.cuda.mem_get_info()[0] == free_before, "the call changed the device's free memory"
+        assert rel_err(to_host_f64(got), to_host_f64(want)) <= tol_for("bf16")
+        oracle = ref.ikbo_linear(co, d["XR"], d["XC"], d["W"], bias=d["bias"], relu=True)
+        assert rel_err(to_host_f64(got), oracle) <= tol_for("bf16")
     rocs.last_device_status()
 
 
