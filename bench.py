@@ -6,8 +6,17 @@ candidates, 768 -> 1024 -> 1024 -> 256, first layer split 512 | 256 between requ
 features): segment plan, request half, candidate half with the in-kernel broadcast, and the two
 plain layers.  `value` is candidates scored per second over all ranks with inputs resident in HBM;
 `e2e` is the same step from pinned host buffers (inputs copied in, scores copied out every step).
-Extra keys report each layer against its own roofline, and the attention (configuration 3) and
-interaction (configuration 4) kernels on their own workloads.
+`roofline` describes the IKBO layer of that step (layer 1: request half + candidate half);
+`dominant_launch` the launch with the largest share of the step.  Extra keys report every layer against
+its own roofline and the other IKBO kernels on their own workloads (attention: configuration 3,
+n_q = 32 / 64 query tokens; interaction, projected FM, group norm: configuration 4 / 2 shapes;
+configuration 5: all three calls), each with a materialised-broadcast GPU comparator and with the cost
+of a fresh segment plan; `summary`, the last key, repeats the headline figures in compact form.
+
+With --gpus N > 1 and no torchrun environment the script starts itself under torch.distributed.run.
+The global batch is N copies of the configuration's requests, split by request over the ranks with
+`sharding.shard_batch` (weights replicated, no collective on the data path, NCCL only for the timing
+barrier and the max over ranks): weak scaling.
 
     python bench.py [--gpus N] [--steps K] [--warmup W] [--impl rocs|reference]
 
@@ -29,7 +38,7 @@ ROOT = os.path.dirname(os.path.abspath(__file__))
 if ROOT not in sys.path:
     sys.path.insert(0, ROOT)
 
-from paper_2607_27744_b200 import workloads as wl  # noqa: E402
+from paper_2607_27744_b200 import sharding, workloads as wl  # noqa: E402
 
 METRIC = "candidates scored/sec per IKBO layer (bf16, 1 B200) and % of roofline"
 UNIT = "candidates/s"
@@ -63,7 +72,7 @@ class ClockSampler:
         try:
             self.proc = subprocess.Popen(
                 ["nvidia-smi", f"--id={self.index}", f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits",
-                 "-lms", "100"], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+                 "-lms", "25"], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
             self.thread = threading.Thread(target=self._read, daemon=True)
             self.thread.start()
         except OSError:
@@ -72,7 +81,7 @@ class ClockSampler:
 
     def _read(self):
         for line in self.proc.stdout:
-            self.rows.append([c.strip() for c in line.split(",")])
+            self.rows.append((time.time(), [c.strip() for c in line.split(",")]))
 
     def __exit__(self, *exc):
         if self.proc:
@@ -83,10 +92,13 @@ class ClockSampler:
                 self.proc.kill()
             self.thread.join(timeout=5)
 
-    def summary(self):
+    def summary(self, t0=None, t1=None):
+        """Median SM clock and the throttle reasons seen between host times t0 and t1 (all samples if None)."""
         sm, mx, reasons = [], [], set()
         names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
-        for r in self.rows:
+        for ts, r in self.rows:
+            if t0 is not None and not (t0 <= ts <= t1):
+                continue
             try:
                 sm.append(float(r[0]))
                 mx.append(float(r[1]))
@@ -167,7 +179,20 @@ def run_reference(args):
 # --------------------------------------------------------------------------------------------
 # CUDA arm
 # --------------------------------------------------------------------------------------------
+def relaunch_under_torchrun(args):
+    """`python bench.py --gpus N` without a torchrun environment: start N ranks of this script."""
+    import socket
+    with socket.socket() as sk:
+        sk.bind(("127.0.0.1", 0))
+        port = sk.getsockname()[1]
+    cmd = [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", f"--nproc-per-node={args.gpus}",
+           "--master-addr", "127.0.0.1", "--master-port", str(port), os.path.abspath(__file__)] + sys.argv[1:]
+    os.execv(sys.executable, cmd)
+
+
 def run_rocs(args):
+    if args.gpus > 1 and "WORLD_SIZE" not in os.environ:
+        relaunch_under_torchrun(args)
     import torch
     from paper_2607_27744_b200 import binding as rocs
 
@@ -183,8 +208,15 @@ def run_rocs(args):
     peaks = measured_peaks()
     cfg = wl.CONFIGS[2]
     data = host_inputs(cfg)
-    co = data["co"]
+    # Requests are independent units (Eq. 1 / Eq. 11).  The global batch is `world` copies of the
+    # configuration's requests; every rank scores the shard sharding.shard_batch gives it (equal-cost
+    # requests: each shard has the single-GPU size), no collective on the data path (weak scaling).
+    co_one = data["co"]
+    shard = sharding.shard_batch(sharding.replicate_offsets(co_one, world), world, rank)
+    co = shard.cand_offsets
     N = int(co[-1])
+    xr_host = data["lin"]["XR"][shard.requests % cfg.R]
+    xc_host = data["lin"]["XC"][shard.cand_rows % int(co_one[-1])]
 
     def dev(a):
         t = torch.from_numpy(np.ascontiguousarray(a))
@@ -194,14 +226,12 @@ def run_rocs(args):
         t = torch.from_numpy(np.ascontiguousarray(a))
         return (t.view(torch.bfloat16) if a.dtype == np.uint16 else t).pin_memory()
 
-    # Requests are independent units (Eq. 1 / Eq. 11): every rank scores its own batch of the same
-    # shape, no collective on the data path (weak scaling).
     W1 = dev(data["lin"]["W"])
     W2, W3 = (dev(w) for w in data["ws"])
     W1_cr, W1_cc = W1[:, :cfg.d_req], W1[:, cfg.d_req:]
     co_dev = dev(co)
-    XR_sets = [dev(data["lin"]["XR"]) for _ in range(N_SETS)]
-    XC_sets = [dev(data["lin"]["XC"]) for _ in range(N_SETS)]
+    XR_sets = [dev(xr_host) for _ in range(N_SETS)]
+    XC_sets = [dev(xc_host) for _ in range(N_SETS)]
     h1 = [torch.empty((N, 1024), dtype=torch.bfloat16, device="cuda") for _ in range(N_SETS)]
     h2 = [torch.empty((N, 1024), dtype=torch.bfloat16, device="cuda") for _ in range(N_SETS)]
     y = [torch.empty((N, 256), dtype=torch.bfloat16, device="cuda") for _ in range(N_SETS)]
@@ -234,10 +264,6 @@ def run_rocs(args):
             dist.barrier()
         torch.cuda.synchronize()
 
-    def ms_estimate(a, b):
-        torch.cuda.synchronize()
-        return a.elapsed_time(b)
-
     def max_over_ranks(ms):
         if dist is None:
             return ms
@@ -254,22 +280,37 @@ def run_rocs(args):
     # region, on the stream the kernels run on (they cost a few hundred ns each)
     marks = [[torch.cuda.Event(enable_timing=True) for _ in range(5)] for _ in range(args.steps)]
     with ClockSampler(local) as clocks:
+        time.sleep(0.06)                   # one sample of the idle GPU in front of the region
+        t_host0 = time.time()
         e0.record()
         for i in range(args.steps):
             step(i, marks=marks[i])
         e1.record()
         barrier()
-        if ms_estimate(e0, e1) < 600.0:   # keep the same load running until a few clock samples exist
-            t_end = time.time() + 0.7
+        t_host1 = time.time()
+        clock_summary = clocks.summary(t_host0, t_host1)
+        clock_summary["sampled"] = "during the timed steps"
+        if clock_summary["samples"] < 3:
+            # A region of a few milliseconds ends before nvidia-smi reports once: the same step keeps
+            # running for 0.7 s and the clocks are read there (load and clocks of the timed steps,
+            # sampled right behind them).
+            t_pad0 = time.time()
             k = 0
-            while time.time() < t_end:
+            while time.time() < t_pad0 + 0.7:
                 step(k)
                 k += 1
             torch.cuda.synchronize()
+            clock_summary = clocks.summary(t_pad0, time.time())
+            clock_summary["sampled"] = "the timed region is too short to sample: same step repeated for 0.7 s right after it"
     ms = max_over_ranks(e0.elapsed_time(e1))
     rocs.last_device_status()
     ms_per_step = ms / args.steps
     value = world * N / (ms_per_step * 1e-3)
+    # A kernel timed in a region of under a second runs at burst clocks: its tensor roof is the burst
+    # measurement; only a seconds-long region is held against the sustained (power-capped) one.
+    sustained_region = ms >= 1000.0
+    tensor_peak = peaks["tflops_sustained"] if sustained_region else peaks["tflops_burst"]
+    tensor_peak_name = ("sustained" if sustained_region else "burst") + f" (timed region {ms:.0f} ms)"
 
     # ---- per-layer durations inside the timed region ------------------------------------------
     def span(a, b):
@@ -290,8 +331,8 @@ def run_rocs(args):
     torch.cuda.synchronize()
     warm = [span_median(warm_marks, a, a + 1) for a in (1, 2, 3)]
 
-    def time_call(fn, reps=20):
-        for i in range(3):
+    def time_call(fn, reps=20, warm=3):
+        for i in range(warm):
             fn(i)
         torch.cuda.synchronize()
         a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
@@ -305,17 +346,16 @@ def run_rocs(args):
     t_plan = time_call(lambda i: rocs.plan_create(co_dev, co).close())
 
     def layer(name, t, flops, nbytes, traffic):
-        # These durations come from inside the long timed step, so a tensor-bound layer is held
-        # against the SUSTAINED measured bf16 peak (the burst figure is given beside it).
         t_hbm = nbytes / (peaks["hbm_gbs"] * 1e9)
-        t_tc = flops / (peaks["tflops_sustained"] * 1e12)
+        t_tc = flops / (tensor_peak * 1e12)
         bound = "hbm" if t_hbm >= t_tc else "tensor"
         ach = nbytes / t / 1e9 if bound == "hbm" else flops / t / 1e12
-        peak = peaks["hbm_gbs"] if bound == "hbm" else peaks["tflops_sustained"]
+        peak = peaks["hbm_gbs"] if bound == "hbm" else tensor_peak
         return {"layer": name, "us": t * 1e6, "cand_per_s": N / t, "bound": bound, "achieved": ach, "peak": peak,
                 "unit": "GB/s" if bound == "hbm" else "TFLOP/s", "frac": ach / peak,
                 "tflops": flops / t / 1e12, "gbs": nbytes / t / 1e9,
                 "frac_of_burst_tensor_peak": flops / t / 1e12 / peaks["tflops_burst"],
+                "frac_of_sustained_tensor_peak": flops / t / 1e12 / peaks["tflops_sustained"],
                 "algorithmic_bytes": nbytes, "traffic": traffic}
 
     bf = 2
@@ -328,13 +368,15 @@ def run_rocs(args):
         layer("cfg2.L3 linear 1024->256", t_l3, 2.0 * N * 1024 * 256, N * 1024 * bf + N * 256 * bf + 256 * 1024 * bf,
               NCU_TRAFFIC["L3"]),
     ]
-    dominant = max(layers, key=lambda l: l["us"])
-    roofline = {"kernel": dominant["layer"], "bound": dominant["bound"], "achieved": dominant["achieved"],
-                "peak": dominant["peak"], "unit": dominant["unit"], "frac": dominant["frac"],
-                "traffic": dominant["traffic"],
-                "peak_source": "of " + peaks["source"] + (" (sustained; timed inside the step)"
-                                                          if dominant["bound"] == "tensor" else ""),
+
+    def roofline_of(lay):
+        return {"kernel": lay["layer"], "bound": lay["bound"], "achieved": lay["achieved"], "peak": lay["peak"],
+                "unit": lay["unit"], "frac": lay["frac"], "traffic": lay["traffic"], "us": lay["us"],
+                "peak_source": "of " + peaks["source"] + (", tensor peak: " + tensor_peak_name if lay["bound"] == "tensor" else ""),
                 "timed": "CUDA events between the calls of every timed step"}
+
+    roofline = roofline_of(layers[0])                          # the IKBO layer of the metric
+    dominant = roofline_of(max(layers, key=lambda l: l["us"]))  # the launch with the largest share of the step
 
     # ---- materialised-broadcast GPU path for the IKBO layer (reference point) ------------------
     counts_dev = dev(np.diff(co).astype(np.int64))
@@ -350,17 +392,12 @@ def run_rocs(args):
         lay["us_median"] = med * 1e6            # median over the timed steps (rotating sets: cold L2)
         lay["us_warm_l2"] = w * 1e6             # median of 30 steps on one buffer set
 
-    # ---- attention and interaction kernels on their own workloads ----------------------------
-    extra = []
-    if not args.skip_extra:
-        extra = bench_other_ops(torch, rocs, peaks, dev, time_call, args.extra.split(","))
-
     # ---- end to end from pinned host buffers ------------------------------------------------
     # Every step copies its inputs from pinned host memory and reads its scores back.  The three
     # phases of consecutive steps are pipelined on three streams (copy-in of step i+1 and copy-out of
     # step i-1 run beside the kernels of step i), with two sets of device input buffers and of host
     # output buffers; every step still moves all of its bytes inside the timed region.
-    XR_h, XC_h, co_h = pinned(data["lin"]["XR"]), pinned(data["lin"]["XC"]), pinned(co)
+    XR_h, XC_h, co_h = pinned(xr_host), pinned(xc_host), pinned(co)
     y_h = [torch.empty((N, 256), dtype=torch.bfloat16).pin_memory() for _ in range(2)]
     in_d = [(torch.empty_like(XR_sets[0]), torch.empty_like(XC_sets[0]), torch.empty_like(co_dev)) for _ in range(2)]
     s_in, s_cmp, s_out = torch.cuda.Stream(), torch.cuda.Stream(), torch.cuda.Stream()
@@ -403,7 +440,16 @@ def run_rocs(args):
     e2e_ms = max_over_ranks(e0.elapsed_time(e1)) / args.steps
     h2d = XR_h.numel() * 2 + XC_h.numel() * 2 + co_h.numel() * 4
     d2h = y_h[0].numel() * 2
+    del XR_sets, XC_sets, h1, h2, y, in_d, y_h, XR_h, XC_h
+    torch.cuda.empty_cache()
 
+    # ---- the other IKBO kernels on their own workloads (rank 0; the data path has no collective) ----
+    extra = []
+    if not args.skip_extra and rank == 0:
+        extra = bench_other_ops(torch, rocs, peaks, dev, time_call, args.extra.split(","))
+    barrier()
+    if dist is not None:
+        dist.destroy_process_group()
     if rank != 0:
         return
     cpu = None
@@ -411,33 +457,54 @@ def run_rocs(args):
         rate, threads, dt, n = sized_oracle_run(data)
         cpu = {"value": rate, "unit": UNIT, "cores": threads, "kind": "oracle",
                "sample": f"{n} evenly spaced candidates of the workload, all three layers, {dt:.1f} s"}
+
+    def brief(l):
+        out = {"us": round(l["us"], 1)}
+        for k_in, k_out in (("frac", "frac"), ("frac_hbm", "frac_hbm"), ("frac_tensor", "frac_tensor_burst"),
+                            ("frac_of_exp_unit_peak_at_max_clock", "frac_exp_unit"),
+                            ("speedup_vs_materialised", "x_materialised"), ("us_with_fresh_plan", "us_fresh_plan")):
+            if k_in in l and l[k_in] is not None:
+                out[k_out] = round(l[k_in], 3 if "frac" in k_out else 1)
+        return out
+
+    summary = {"cfg2.L1": brief(layers[0]) | {"bound": layers[0]["bound"]},
+               "cfg2.L2": brief(layers[1]) | {"bound": layers[1]["bound"]},
+               "cfg2.L3": brief(layers[2]) | {"bound": layers[2]["bound"]}}
+    for l in extra:
+        summary[l["key"]] = brief(l)
     print(json.dumps({
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
         "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
         "dtype": "bf16", "data": "synthetic",
         "config": {"workload": WORKLOAD, "l2": f"{N_SETS} rotating input/activation sets, larger than L2",
-                   "step": "plan + request half + candidate half (in-kernel broadcast) + 2 plain layers"},
-        "clocks": clocks.summary(),
+                   "step": "plan + request half + candidate half (in-kernel broadcast) + 2 plain layers",
+                   "sharding": f"global batch = {world} x the workload's requests, split by request "
+                               f"(sharding.shard_batch), {shard.requests.size} requests / {N} candidates per rank"},
+        "clocks": clock_summary,
         "e2e": {"value": world * N / (e2e_ms * 1e-3), "unit": UNIT, "h2d_bytes_per_step": h2d,
                 "d2h_bytes_per_step": d2h, "ms_per_step": e2e_ms},
         "gpu_launches": launches_per_step * args.steps,
         "roofline": roofline,
+        "dominant_launch": dominant,
         "cpu_baseline": cpu,
         "layers": layers,
         "plan_us": t_plan * 1e6, "plan_us_in_step": t_plan_in * 1e6,
         "other_ikbo_layers": extra,
+        "summary": summary,
     }))
 
 
-def bench_other_ops(torch, rocs, peaks, dev, time_call, which=("dca", "glm")):
-    """Attention on configuration 3 and interaction on configuration 4, one layer each."""
+def bench_other_ops(torch, rocs, peaks, dev, time_call, which):
+    """The other IKBO kernels, one layer each, on their own workloads."""
     out = []
     if "dca" in which:
         out.append(bench_dca(torch, rocs, peaks, dev, time_call))
+    if "nq" in which:
+        out.append(bench_dca_nq(torch, rocs, peaks, dev, time_call, 32))
+    if "nq64" in which:
+        out.append(bench_dca_nq(torch, rocs, peaks, dev, time_call, 64))
     if "glm" in which:
         out.append(bench_glm(torch, rocs, peaks, dev, time_call))
-    if "nq" in which:
-        out.append(bench_dca_nq(torch, rocs, peaks, dev, time_call))
     if "fm" in which:
         out.append(bench_fm(torch, rocs, peaks, dev, time_call))
     if "norm" in which:
@@ -455,12 +522,21 @@ def materialised_linear(torch, XR, XC, W, counts_dev, relu=True):
     return torch.relu_(y) if relu else y
 
 
-def materialised_dca(torch, Q, K, V, co, so, chunk_bytes=4 << 30):
+def materialised_linear_chunked(torch, XR, XC, W, row2req, chunk=1 << 18):
+    """The same in candidate chunks, for batches whose materialised input does not fit at once."""
+    for a in range(0, XC.shape[0], chunk):
+        b = min(XC.shape[0], a + chunk)
+        u = torch.cat([XR[row2req[a:b]], XC[a:b]], dim=1)
+        y = u @ W.t()
+    return y
+
+
+def materialised_dca(torch, Q, K, V, co, so, chunk_bytes=4 << 30, requests=None):
     """Candidate-batched copies of K/V, then library attention (Section 4.3, second paragraph),
-    request by request in chunks so the copies fit in memory."""
+    request by request in chunks so the copies fit in memory; `requests` restricts it to a sample."""
     N, n_q, H, dh = Q.shape
     O = torch.empty_like(Q)
-    for r in range(len(co) - 1):
+    for r in (range(len(co) - 1) if requests is None else requests):
         c0, c1, s0, s1 = int(co[r]), int(co[r + 1]), int(so[r]), int(so[r + 1])
         if c1 == c0 or s1 == s0:
             continue
@@ -487,27 +563,57 @@ def materialised_glm(torch, XR, XC, W, counts_dev, n_r, n_ro):
     return torch.matmul(Wm, G)
 
 
+def materialised_glm_rows_chunked(torch, XR, XC, row2req, chunk=1 << 17):
+    """Candidate rows of the masked interaction from the materialised X, in candidate chunks."""
+    for a in range(0, XC.shape[0], chunk):
+        b = min(XC.shape[0], a + chunk)
+        X = torch.cat([XR[row2req[a:b]], XC[a:b]], dim=1)
+        G = torch.bmm(XC[a:b], X.transpose(1, 2))
+    return G
+
+
+def with_fresh_plan(rocs, time_call, co_dev, co, call, reps=5):
+    """The same call when the batch is new: segment plan (request ids, work list) built in front of it."""
+    def once(i):
+        plan = rocs.plan_create(co_dev, co)
+        call(plan)
+        plan.close()
+    return time_call(once, reps=reps)
+
+
+def dca_record(key, name, cfg, N, co, so, t, t_fresh, t_mat, peaks, rows_per_cand=1, mat_note=None):
+    pairs = float(np.sum(np.diff(co).astype(np.float64) * np.diff(so))) * rows_per_cand
+    flops = 4.0 * pairs * cfg.H * cfg.dh
+    rec = {"key": key, "layer": name, "N": N, "us": t * 1e6, "us_with_fresh_plan": t_fresh * 1e6,
+           "cand_per_s": N / t, "tflops": flops / t / 1e12,
+           "frac_tensor": flops / t / 1e12 / peaks["tflops_burst"],
+           "frac_tensor_sustained": flops / t / 1e12 / peaks["tflops_sustained"],
+           "exps_per_s": pairs * cfg.H / t,
+           "frac_of_exp_unit_peak_at_max_clock": pairs * cfg.H / t / (148 * 16 * 1.965e9),
+           "bound": "tensor (nominal: 4 L H dh flop per candidate against the burst bf16 peak); at dh = 64 the "
+                    "exponential unit (16 ex2/clk/SM, one per 256 tensor flops) is the tighter ceiling"}
+    if t_mat is not None:
+        rec["materialised_broadcast_gpu_us"] = t_mat * 1e6
+        rec["speedup_vs_materialised"] = t_mat / t
+        if mat_note:
+            rec["materialised_note"] = mat_note
+    return rec
+
+
 def bench_dca(torch, rocs, peaks, dev, time_call):
     # configuration 3: one DCA layer
     cfg = wl.CONFIGS[3]
     co, so = wl.cand_offsets(cfg), wl.seq_offsets(cfg)
     N = int(co[-1])
     d = wl.dca_inputs(cfg, co, so)
-    plan = rocs.plan_create(dev(co), co)
+    co_dev = dev(co)
+    plan = rocs.plan_create(co_dev, co)
     Q, K, V, sod = dev(d["Q"]), dev(d["K"]), dev(d["V"]), dev(so)
     O = torch.empty_like(Q)
-    t = time_call(lambda i: rocs.dca_attention(plan, Q, K, V, sod, out=O), reps=5)
-    pairs = float(np.sum(np.diff(co).astype(np.float64) * np.diff(so)))
-    flops = 4.0 * pairs * cfg.H * cfg.dh
-    nbytes = (2 * Q.numel() + 2 * K.numel()) * 2
-    t_mat = time_call(lambda i: materialised_dca(torch, Q, K, V, co, so), reps=1)
-    return {"layer": "cfg3 dca_attention (R=64, L=2048, 8x64)", "N": N, "us": t * 1e6, "cand_per_s": N / t,
-            "materialised_broadcast_gpu_us": t_mat * 1e6, "speedup_vs_materialised": t_mat / t,
-            "tflops": flops / t / 1e12, "frac_tensor": flops / t / 1e12 / peaks["tflops_burst"],
-            "gbs": nbytes / t / 1e9, "exps_per_s": pairs * cfg.H / t,
-            "bound": "tensor (nominal); the exponential unit (16 ex2/clk/SM) is the tighter ceiling at dh = 64",
-            "frac_of_exp_unit_peak_at_max_clock": pairs * cfg.H / t / (148 * 16 * 1.965e9),
-            "frac_tensor_sustained": flops / t / 1e12 / peaks["tflops_sustained"]}
+    t = time_call(lambda i: rocs.dca_attention(plan, Q, K, V, sod, out=O), reps=10)
+    t_fresh = with_fresh_plan(rocs, time_call, co_dev, co, lambda pl: rocs.dca_attention(pl, Q, K, V, sod, out=O), reps=10)
+    t_mat = time_call(lambda i: materialised_dca(torch, Q, K, V, co, so), reps=1, warm=1)
+    return dca_record("cfg3.dca", "cfg3 dca_attention (R=64, L=2048, 8x64)", cfg, N, co, so, t, t_fresh, t_mat, peaks)
 
 
 def bench_dca_nq(torch, rocs, peaks, dev, time_call, n_q=32):
@@ -519,15 +625,16 @@ def bench_dca_nq(torch, rocs, peaks, dev, time_call, n_q=32):
     co, so = wl.offsets_from_counts(counts.tolist()), wl.seq_offsets(base)
     N = int(co[-1])
     d = wl.dca_inputs(cfg, co, so)
-    plan = rocs.plan_create(dev(co), co)
+    co_dev = dev(co)
+    plan = rocs.plan_create(co_dev, co)
     Q, K, V, sod = dev(d["Q"]), dev(d["K"]), dev(d["V"]), dev(so)
     O = torch.empty_like(Q)
-    t = time_call(lambda i: rocs.dca_attention(plan, Q, K, V, sod, out=O), reps=5)
-    pairs = float(np.sum(np.diff(co).astype(np.float64) * np.diff(so))) * n_q
-    flops = 4.0 * pairs * cfg.H * cfg.dh
-    return {"layer": f"cfg3 dca_attention with n_q={n_q} query tokens per candidate (R=64, L=2048, 8x64)", "N": N,
-            "us": t * 1e6, "cand_per_s": N / t, "query_rows_per_s": N * n_q / t, "tflops": flops / t / 1e12,
-            "frac_tensor": flops / t / 1e12 / peaks["tflops_burst"], "exps_per_s": pairs * cfg.H / t}
+    t = time_call(lambda i: rocs.dca_attention(plan, Q, K, V, sod, out=O), reps=10)
+    t_fresh = with_fresh_plan(rocs, time_call, co_dev, co, lambda pl: rocs.dca_attention(pl, Q, K, V, sod, out=O), reps=10)
+    rec = dca_record(f"cfg3.dca_nq{n_q}", f"cfg3 dca_attention with n_q={n_q} query tokens per candidate (R=64, L=2048, 8x64)",
+                     cfg, N, co, so, t, t_fresh, None, peaks, rows_per_cand=n_q)
+    rec["query_rows_per_s"] = N * n_q / t
+    return rec
 
 
 def bench_glm(torch, rocs, peaks, dev, time_call):
@@ -536,22 +643,25 @@ def bench_glm(torch, rocs, peaks, dev, time_call):
     co = wl.cand_offsets(cfg)
     N = int(co[-1])
     d = wl.glm_inputs(cfg, co)
-    plan4 = rocs.plan_create(dev(co), co)
+    co_dev = dev(co)
+    plan4 = rocs.plan_create(co_dev, co)
     XR, XC, W = dev(d["XR"]), dev(d["XC"]), dev(d["W"])
     n = cfg.n_r + cfg.n_c
     outs = {"OC": torch.empty((N, cfg.n_co, n), dtype=torch.bfloat16, device="cuda"),
             "OR": torch.empty((cfg.R, cfg.n_ro, n), dtype=torch.bfloat16, device="cuda")}
     ws = torch.empty(rocs.glm_interaction_workspace(plan4, cfg.n_r, cfg.n_c, cfg.n_co), dtype=torch.uint8, device="cuda")
-    t = time_call(lambda i: rocs.glm_interaction(plan4, XR, XC, W, cfg.n_ro, cfg.n_co, want_raw=False, workspace=ws,
-                                                 outs=outs), reps=10)
+    call = lambda pl: rocs.glm_interaction(pl, XR, XC, W, cfg.n_ro, cfg.n_co, want_raw=False, workspace=ws, outs=outs)
+    t = time_call(lambda i: call(plan4), reps=10)
+    t_fresh = with_fresh_plan(rocs, time_call, co_dev, co, call, reps=10)
     nbytes = XC.numel() * 2 + outs["OC"].numel() * 2 + XR.numel() * 2
     flops = N * (2.0 * cfg.n_c * n * cfg.d_emb + 2.0 * cfg.n_co * cfg.n_c * n)
     counts_dev = dev(np.diff(co).astype(np.int64))
     t_mat = time_call(lambda i: materialised_glm(torch, XR, XC, W, counts_dev, cfg.n_r, cfg.n_ro), reps=3)
-    return {"layer": "cfg4 glm_interaction 32+16 x128, 48->16 compression (OC only)", "N": N, "us": t * 1e6,
+    return {"key": "cfg4.glm", "layer": "cfg4 glm_interaction 32+16 x128, 48->16 compression (OC only)", "N": N,
+            "us": t * 1e6, "us_with_fresh_plan": t_fresh * 1e6,
             "materialised_broadcast_gpu_us": t_mat * 1e6, "speedup_vs_materialised": t_mat / t,
             "cand_per_s": N / t, "gbs": nbytes / t / 1e9, "frac_hbm": nbytes / t / 1e9 / peaks["hbm_gbs"],
-            "tflops": flops / t / 1e12,
+            "tflops": flops / t / 1e12, "bound": "hbm",
             "note": "input (537 MB) is larger than L2; same buffers every iteration"}
 
 
@@ -569,20 +679,24 @@ def bench_fm(torch, rocs, peaks, dev, time_call):
     co = wl.cand_offsets(cfg)
     N = int(co[-1])
     d = wl.glm_inputs(cfg, co)
-    plan4 = rocs.plan_create(dev(co), co)
+    co_dev = dev(co)
+    plan4 = rocs.plan_create(co_dev, co)
     XR, XC, P = dev(d["XR"]), dev(d["XC"]), dev(wl.fm_projection_weight(cfg, k))
     outs = {"FC": torch.empty((N, cfg.n_c, k), dtype=torch.bfloat16, device="cuda"),
             "FR": torch.empty((cfg.R, cfg.n_r, k), dtype=torch.bfloat16, device="cuda")}
     ws = torch.empty(rocs.glm_fm_projection_workspace(plan4, cfg.d_emb, k), dtype=torch.uint8, device="cuda")
-    t = time_call(lambda i: rocs.glm_fm_projection(plan4, XR, XC, P, workspace=ws, outs=outs), reps=10)
+    call = lambda pl: rocs.glm_fm_projection(pl, XR, XC, P, workspace=ws, outs=outs)
+    t = time_call(lambda i: call(plan4), reps=10)
+    t_fresh = with_fresh_plan(rocs, time_call, co_dev, co, call, reps=10)
     nbytes = XC.numel() * 2 + outs["FC"].numel() * 2 + XR.numel() * 2
     flops = N * 4.0 * cfg.n_c * cfg.d_emb * k
     counts_dev = dev(np.diff(co).astype(np.int64))
     t_mat = time_call(lambda i: materialised_fm(torch, XR, XC, P, counts_dev, cfg.n_r), reps=3)
-    return {"layer": "cfg4 shapes glm_fm_projection 32+16 x128 -> k=16", "N": N, "us": t * 1e6,
+    return {"key": "cfg4.fm", "layer": "cfg4 shapes glm_fm_projection 32+16 x128 -> k=16", "N": N, "us": t * 1e6,
+            "us_with_fresh_plan": t_fresh * 1e6,
             "materialised_broadcast_gpu_us": t_mat * 1e6, "speedup_vs_materialised": t_mat / t,
             "cand_per_s": N / t, "gbs": nbytes / t / 1e9, "frac_hbm": nbytes / t / 1e9 / peaks["hbm_gbs"],
-            "tflops": flops / t / 1e12,
+            "tflops": flops / t / 1e12, "bound": "hbm",
             "note": "input (537 MB) is larger than L2; same buffers every iteration"}
 
 
@@ -597,30 +711,36 @@ def bench_norm(torch, rocs, peaks, dev, time_call):
     t = time_call(lambda i: rocs.group_norm(X, gamma, None, 1e-6, rocs.NORM_RMS, out=Y), reps=20)
     nbytes = 2 * X.numel() * 2
     t_lib = time_call(lambda i: torch.nn.functional.rms_norm(X, (cfg.d_out,), gamma, eps=1e-6), reps=20)
-    return {"layer": "cfg2 activations group_norm (RMSNorm, 131072 x 1024)", "N": N, "us": t * 1e6, "cand_per_s": N / t,
-            "gbs": nbytes / t / 1e9, "frac_hbm": nbytes / t / 1e9 / peaks["hbm_gbs"], "torch_rms_norm_us": t_lib * 1e6,
+    return {"key": "cfg2.norm", "layer": "cfg2 activations group_norm (RMSNorm, 131072 x 1024)", "N": N, "us": t * 1e6,
+            "cand_per_s": N / t, "gbs": nbytes / t / 1e9, "frac_hbm": nbytes / t / 1e9 / peaks["hbm_gbs"],
+            "torch_rms_norm_us": t_lib * 1e6, "bound": "hbm",
             "note": "input and output (537 MB) are larger than L2"}
 
 
 def bench_cfg5(torch, rocs, peaks, dev, time_call):
-    """Configuration 5 (skewed, Zipf candidate counts): the three calls timed independently."""
+    """Configuration 5 (skewed, Zipf candidate counts): the three calls timed independently, each
+    against a materialised-broadcast GPU path."""
     cfg = wl.CONFIGS[5]
     co, so = wl.cand_offsets(cfg), wl.seq_offsets(cfg)
     N = int(co[-1])
-    plan = rocs.plan_create(dev(co), co)
+    co_dev = dev(co)
+    plan = rocs.plan_create(co_dev, co)
     out = []
     g = torch.Generator(device="cuda").manual_seed(5)
     rnd = lambda *shape: torch.randn(*shape, generator=g, device="cuda", dtype=torch.float32).to(torch.bfloat16)
+    row2req = torch.repeat_interleave(torch.arange(cfg.R, device="cuda"), dev(np.diff(co).astype(np.int64)))
     # linear 768|256 -> 1024
     XR, XC = rnd(cfg.R, cfg.d_req), rnd(N, cfg.d_cand)
     W = (rnd(cfg.d_out, cfg.d_req + cfg.d_cand).float() / 32).to(torch.bfloat16)
     Y = torch.empty((N, cfg.d_out), dtype=torch.bfloat16, device="cuda")
     ws = torch.empty(rocs.ikbo_linear_workspace(plan, cfg.d_out), dtype=torch.uint8, device="cuda")
-    t = time_call(lambda i: rocs.ikbo_linear(plan, XR, XC, W[:, :cfg.d_req], W[:, cfg.d_req:], out=Y, workspace=ws), reps=5)
+    call = lambda pl: rocs.ikbo_linear(pl, XR, XC, W[:, :cfg.d_req], W[:, cfg.d_req:], out=Y, workspace=ws)
+    t = time_call(lambda i: call(plan), reps=5)
+    t_fresh = with_fresh_plan(rocs, time_call, co_dev, co, call)
     nbytes = (XC.numel() + Y.numel() + XR.numel() + W.numel()) * 2
-    counts_dev = dev(np.diff(co).astype(np.int64))
-    t_mat = time_call(lambda i: materialised_linear(torch, XR, XC, W, counts_dev, relu=False), reps=2)
-    out.append({"layer": "cfg5 ikbo_linear 768|256->1024 (Zipf segments)", "N": N, "us": t * 1e6, "cand_per_s": N / t,
+    t_mat = time_call(lambda i: materialised_linear_chunked(torch, XR, XC, W, row2req), reps=2, warm=1)
+    out.append({"key": "cfg5.linear", "layer": "cfg5 ikbo_linear 768|256->1024 (Zipf segments)", "N": N, "us": t * 1e6,
+                "us_with_fresh_plan": t_fresh * 1e6, "cand_per_s": N / t, "bound": "hbm",
                 "gbs": nbytes / t / 1e9, "frac_hbm": nbytes / t / 1e9 / peaks["hbm_gbs"],
                 "materialised_broadcast_gpu_us": t_mat * 1e6, "speedup_vs_materialised": t_mat / t})
     del XC, Y
@@ -629,22 +749,33 @@ def bench_cfg5(torch, rocs, peaks, dev, time_call):
     Q, K, V = rnd(N, 1, cfg.H, cfg.dh), rnd(T, cfg.H, cfg.dh), rnd(T, cfg.H, cfg.dh)
     O = torch.empty_like(Q)
     sod = dev(so)
-    t = time_call(lambda i: rocs.dca_attention(plan, Q, K, V, sod, out=O), reps=3)
-    pairs = float(np.sum(np.diff(co).astype(np.float64) * np.diff(so)))
-    flops = 4.0 * pairs * cfg.H * cfg.dh
-    out.append({"layer": "cfg5 dca_attention (Zipf segments, L in [256,1024], 8x64)", "N": N, "us": t * 1e6,
-                "cand_per_s": N / t, "tflops": flops / t / 1e12, "frac_tensor": flops / t / 1e12 / peaks["tflops_burst"],
-                "exps_per_s": pairs * cfg.H / t})
+    call = lambda pl: rocs.dca_attention(pl, Q, K, V, sod, out=O)
+    t = time_call(lambda i: call(plan), reps=3)
+    t_fresh = with_fresh_plan(rocs, time_call, co_dev, co, call, reps=3)
+    # the materialised path copies K and V once per candidate (about 2 TB here): timed on every 16th
+    # request and scaled by key-candidate pairs
+    pairs_r = np.diff(co).astype(np.float64) * np.diff(so)
+    sample = list(range(3, cfg.R, 16))
+    t_mat_s = time_call(lambda i: materialised_dca(torch, Q, K, V, co, so, requests=sample), reps=1, warm=0)
+    t_mat = t_mat_s * float(pairs_r.sum() / max(1.0, pairs_r[sample].sum()))
+    out.append(dca_record("cfg5.dca", "cfg5 dca_attention (Zipf segments, L in [256,1024], 8x64)", cfg, N, co, so, t,
+                          t_fresh, t_mat, peaks,
+                          mat_note="measured on every 16th request, scaled by key-candidate pairs"))
     del Q, K, V, O
     # interaction 24 + 8, no compression
     GR, GC = rnd(cfg.R, cfg.n_r, cfg.d_emb), rnd(N, cfg.n_c, cfg.d_emb)
     n = cfg.n_r + cfg.n_c
     outs = {"YC": torch.empty((N, cfg.n_c, n), dtype=torch.bfloat16, device="cuda"),
             "YR": torch.empty((cfg.R, cfg.n_r, n), dtype=torch.bfloat16, device="cuda")}
-    t = time_call(lambda i: rocs.glm_interaction(plan, GR, GC, None, 0, 0, want_raw=True, outs=outs), reps=5)
+    call = lambda pl: rocs.glm_interaction(pl, GR, GC, None, 0, 0, want_raw=True, outs=outs)
+    t = time_call(lambda i: call(plan), reps=5)
+    t_fresh = with_fresh_plan(rocs, time_call, co_dev, co, call)
     nbytes = (GC.numel() + outs["YC"].numel()) * 2
-    out.append({"layer": "cfg5 glm_interaction 24+8 x128 (raw YC)", "N": N, "us": t * 1e6, "cand_per_s": N / t,
-                "gbs": nbytes / t / 1e9, "frac_hbm": nbytes / t / 1e9 / peaks["hbm_gbs"]})
+    t_mat = time_call(lambda i: materialised_glm_rows_chunked(torch, GR, GC, row2req), reps=2, warm=1)
+    out.append({"key": "cfg5.glm", "layer": "cfg5 glm_interaction 24+8 x128 (raw YC)", "N": N, "us": t * 1e6,
+                "us_with_fresh_plan": t_fresh * 1e6, "cand_per_s": N / t, "bound": "hbm",
+                "gbs": nbytes / t / 1e9, "frac_hbm": nbytes / t / 1e9 / peaks["hbm_gbs"],
+                "materialised_broadcast_gpu_us": t_mat * 1e6, "speedup_vs_materialised": t_mat / t})
     return out
 
 
@@ -655,7 +786,8 @@ def main():
     ap.add_argument("--warmup", type=int, default=10)
     ap.add_argument("--impl", default="rocs", choices=["rocs", "reference"])
     ap.add_argument("--skip-extra", action="store_true", help="skip the attention / interaction side measurements")
-    ap.add_argument("--extra", default="dca,glm", help="side measurements to run: dca, nq, glm, fm, norm, cfg5")
+    ap.add_argument("--extra", default="dca,nq,nq64,glm,fm,norm,cfg5",
+                    help="side measurements to run: dca, nq, nq64, glm, fm, norm, cfg5")
     ap.add_argument("--skip-cpu", action="store_true", help="skip the cpu_baseline leg")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "rocs" else args.warmup

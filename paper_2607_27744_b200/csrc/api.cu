@@ -38,6 +38,67 @@ uint32_t* device_status_word() {
   return p;
 }
 
+// Work lists are expanded on the device: the host only adds up the tile counts of the R requests
+// (tile_base, R + 1 integers), every list entry then finds its request by binary search in that
+// prefix array, so a batch with hundreds of thousands of entries costs one small copy and one launch.
+__global__ void expand_tiles_kernel(int32_t R, int32_t total, int32_t cands_per_tile,
+                                    const int32_t* __restrict__ off, const int32_t* __restrict__ tile_base,
+                                    Tile* __restrict__ out) {
+  const int32_t i = blockIdx.x * blockDim.x + threadIdx.x;
+  if (i >= total) return;
+  int32_t lo = 0, hi = R;  // largest r with tile_base[r] <= i
+  while (hi - lo > 1) {
+    const int32_t mid = lo + (hi - lo) / 2;
+    if (tile_base[mid] <= i) lo = mid; else hi = mid;
+  }
+  const int32_t c = off[lo] + (i - tile_base[lo]) * cands_per_tile;
+  out[i] = Tile{lo, c, min(cands_per_tile, off[lo + 1] - c), 0};
+}
+
+// Attention items in the order request, head, tile (or tile pair).
+__global__ void expand_dca_items_kernel(int32_t R, int32_t total, int32_t cands_per_tile, int32_t heads,
+                                        int32_t tiles_per_item, const int32_t* __restrict__ off,
+                                        const int32_t* __restrict__ item_base, DcaItem* __restrict__ out) {
+  const int32_t i = blockIdx.x * blockDim.x + threadIdx.x;
+  if (i >= total) return;
+  int32_t lo = 0, hi = R;  // largest r with item_base[r] * heads <= i
+  while (hi - lo > 1) {
+    const int32_t mid = lo + (hi - lo) / 2;
+    if ((int64_t)item_base[mid] * heads <= i) lo = mid; else hi = mid;
+  }
+  const int32_t per_head = item_base[lo + 1] - item_base[lo];
+  const int32_t local = i - item_base[lo] * heads;
+  const int32_t h = local / per_head, t = local % per_head;
+  const int32_t c = off[lo] + t * tiles_per_item * cands_per_tile, c_end = off[lo + 1];
+  const int32_t a = min(cands_per_tile, c_end - c);
+  const int32_t b = tiles_per_item == 2 ? min(cands_per_tile, c_end - c - a) : 0;
+  out[i] = DcaItem{lo, c, (int16_t)a, (int16_t)b, h};
+}
+
+// Prefix sums of ceil(n_r / per_entry) over the requests, copied to the device.  Returns the total
+// through *total; *base_dev is a stream-ordered allocation the caller frees after its kernel.
+static rocs_status_t upload_entry_base(const rocs_plan* plan, int32_t per_entry, cudaStream_t stream,
+                                       int32_t** base_dev, int64_t* total) {
+  std::vector<int32_t> base((size_t)plan->R + 1);
+  int64_t acc = 0;
+  for (int32_t r = 0; r < plan->R; ++r) {
+    base[r] = (int32_t)acc;
+    const int64_t n = (int64_t)plan->offsets_host[r + 1] - plan->offsets_host[r];
+    acc += (n + per_entry - 1) / per_entry;
+    if (acc > 0x7fffffffLL) return ROCS_ERR_UNSUPPORTED;
+  }
+  base[plan->R] = (int32_t)acc;
+  *total = acc;
+  ROCS_CUDA_TRY(cudaMallocAsync((void**)base_dev, sizeof(int32_t) * base.size(), stream));
+  // Pageable source: the copy is staged before the call returns, so `base` may go away.
+  if (cudaMemcpyAsync(*base_dev, base.data(), sizeof(int32_t) * base.size(), cudaMemcpyHostToDevice, stream) !=
+      cudaSuccess) {
+    cudaFreeAsync(*base_dev, stream);
+    return ROCS_ERR_CUDA;
+  }
+  return ROCS_OK;
+}
+
 rocs_status_t plan_tiles(const rocs_plan* plan, int32_t cands_per_tile, cudaStream_t stream,
                          TileList* out) {
   if (cands_per_tile < 1) return ROCS_ERR_INVALID_ARG;
@@ -47,20 +108,22 @@ rocs_status_t plan_tiles(const rocs_plan* plan, int32_t cands_per_tile, cudaStre
     *out = it->second;
     return ROCS_OK;
   }
-  std::vector<Tile> host;
-  for (int32_t r = 0; r < plan->R; ++r)
-    for (int32_t c = plan->offsets_host[r]; c < plan->offsets_host[r + 1]; c += cands_per_tile)
-      host.push_back(Tile{r, c, std::min(cands_per_tile, plan->offsets_host[r + 1] - c), 0});
   TileList tl;
-  tl.num = (int32_t)host.size();
-  if (tl.num > 0) {
-    ROCS_CUDA_TRY(cudaMallocAsync((void**)&tl.dev, sizeof(Tile) * host.size(), stream));
-    // Pageable source: the copy is staged before the call returns, so `host` may go away.
-    if (cudaMemcpyAsync(tl.dev, host.data(), sizeof(Tile) * host.size(), cudaMemcpyHostToDevice,
-                        stream) != cudaSuccess) {
-      cudaFreeAsync(tl.dev, stream);
-      return ROCS_ERR_CUDA;
+  if (plan->N > 0) {
+    int32_t* base_dev = nullptr;
+    int64_t total = 0;
+    rocs_status_t st = upload_entry_base(plan, cands_per_tile, stream, &base_dev, &total);
+    if (st != ROCS_OK) return st;
+    tl.num = (int32_t)total;
+    cudaError_t e = cudaMallocAsync((void**)&tl.dev, sizeof(Tile) * (size_t)total, stream);
+    if (e == cudaSuccess) {
+      expand_tiles_kernel<<<(unsigned)((total + 255) / 256), 256, 0, stream>>>(plan->R, tl.num, cands_per_tile,
+                                                                              plan->cand_offsets, base_dev, tl.dev);
+      e = cudaGetLastError();
+      if (e != cudaSuccess) cudaFreeAsync(tl.dev, stream);
     }
+    cudaFreeAsync(base_dev, stream);
+    if (e != cudaSuccess) return ROCS_ERR_CUDA;
   }
   plan->tiles[cands_per_tile] = tl;
   *out = tl;
@@ -79,26 +142,27 @@ rocs_status_t plan_dca_items(const rocs_plan* plan, int32_t cands_per_tile, int3
     *out = it->second;
     return ROCS_OK;
   }
-  std::vector<DcaItem> host;
-  for (int32_t r = 0; r < plan->R; ++r) {
-    const int32_t c_begin = plan->offsets_host[r], c_end = plan->offsets_host[r + 1];
-    if (c_begin == c_end) continue;
-    for (int32_t h = 0; h < heads; ++h)
-      for (int32_t c = c_begin; c < c_end; c += tiles_per_item * cands_per_tile) {
-        const int32_t a = std::min(cands_per_tile, c_end - c);
-        const int32_t b = tiles_per_item == 2 ? std::min(cands_per_tile, c_end - c - a) : 0;
-        host.push_back(DcaItem{r, c, (int16_t)a, (int16_t)b, h});
-      }
-  }
   DcaItemList il;
-  il.num = (int32_t)host.size();
-  if (il.num > 0) {
-    ROCS_CUDA_TRY(cudaMallocAsync((void**)&il.dev, sizeof(DcaItem) * host.size(), stream));
-    if (cudaMemcpyAsync(il.dev, host.data(), sizeof(DcaItem) * host.size(), cudaMemcpyHostToDevice, stream) !=
-        cudaSuccess) {
-      cudaFreeAsync(il.dev, stream);
-      return ROCS_ERR_CUDA;
+  if (plan->N > 0) {
+    int32_t* base_dev = nullptr;
+    int64_t per_head = 0;
+    rocs_status_t st = upload_entry_base(plan, cands_per_tile * tiles_per_item, stream, &base_dev, &per_head);
+    if (st != ROCS_OK) return st;
+    const int64_t total = per_head * heads;
+    if (total > 0x7fffffffLL) {
+      cudaFreeAsync(base_dev, stream);
+      return ROCS_ERR_UNSUPPORTED;
     }
+    il.num = (int32_t)total;
+    cudaError_t e = cudaMallocAsync((void**)&il.dev, sizeof(DcaItem) * (size_t)total, stream);
+    if (e == cudaSuccess) {
+      expand_dca_items_kernel<<<(unsigned)((total + 255) / 256), 256, 0, stream>>>(
+          plan->R, il.num, cands_per_tile, heads, tiles_per_item, plan->cand_offsets, base_dev, il.dev);
+      e = cudaGetLastError();
+      if (e != cudaSuccess) cudaFreeAsync(il.dev, stream);
+    }
+    cudaFreeAsync(base_dev, stream);
+    if (e != cudaSuccess) return ROCS_ERR_CUDA;
   }
   plan->dca_items[key] = il;
   *out = il;

@@ -46,3 +46,36 @@ def shard_rows(offsets: np.ndarray, requests: np.ndarray):
     rows = np.concatenate([np.arange(offsets[r], offsets[r + 1]) for r in requests]) if len(requests) else \
         np.zeros(0, np.int64)
     return rows, local.astype(np.int32)
+
+
+def replicate_offsets(offsets: np.ndarray, copies: int) -> np.ndarray:
+    """Offsets of a global batch made of `copies` batches with these offsets, one after the other."""
+    counts = np.diff(np.asarray(offsets, np.int64))
+    out = np.zeros(copies * counts.size + 1, np.int64)
+    np.cumsum(np.tile(counts, copies), out=out[1:])
+    return out
+
+
+class Shard:
+    """What one rank scores of a global batch: its requests (global indices, ascending), the global
+    candidate rows they own (in request order), the rank's own ``cand_offsets``, and the same for the
+    sequence positions when the batch has sequences."""
+
+    def __init__(self, requests, cand_rows, cand_offsets, seq_rows=None, seq_offsets=None):
+        self.requests, self.cand_rows, self.cand_offsets = requests, cand_rows, cand_offsets
+        self.seq_rows, self.seq_offsets = seq_rows, seq_offsets
+
+
+def shard_batch(cand_offsets: np.ndarray, world_size: int, rank: int, seq_offsets: Optional[np.ndarray] = None,
+                c_linear: float = 1.0, c_attn: float = 0.0, c_glm: float = 0.0) -> Shard:
+    """Shard of `rank` when the global batch is split by request over `world_size` ranks (no rank
+    needs anything from another: there is no collective on the data path)."""
+    cand_offsets = np.asarray(cand_offsets, np.int64)
+    lens = None if seq_offsets is None else np.diff(np.asarray(seq_offsets, np.int64))
+    cost = request_cost(np.diff(cand_offsets), lens, c_linear=c_linear, c_attn=c_attn, c_glm=c_glm)
+    mine = partition_requests(cost, world_size)[rank]
+    rows, co_l = shard_rows(cand_offsets, mine)
+    if seq_offsets is None:
+        return Shard(mine, rows, co_l)
+    seq_rows, so_l = shard_rows(seq_offsets, mine)
+    return Shard(mine, rows, co_l, seq_rows, so_l)

@@ -39,6 +39,21 @@ def test_shard_rows_builds_local_offsets():
     assert rows.size == 0 and local.tolist() == [0]
 
 
+def test_replicated_global_batch_shards_into_equal_weak_scaling_pieces():
+    """bench.py --gpus N builds a global batch of N copies of the configuration's requests and gives
+    every rank its shard: equal-cost requests must split into N shards of the single-GPU size that
+    together cover every candidate once."""
+    cfg = wl.CONFIGS[2].with_(R=16)
+    co = wl.cand_offsets(cfg)
+    for world in (1, 2, 4, 8):
+        glob = sharding.replicate_offsets(co, world)
+        assert glob.size == world * cfg.R + 1 and glob[-1] == world * co[-1]
+        shards = [sharding.shard_batch(glob, world, r) for r in range(world)]
+        assert all(sh.requests.size == cfg.R and sh.cand_offsets[-1] == co[-1] for sh in shards)
+        rows = np.concatenate([sh.cand_rows for sh in shards])
+        assert np.array_equal(np.sort(rows), np.arange(glob[-1]))
+
+
 def _worker(rank, world, port, out_q):
     sys.path.insert(0, ROOT)
     from oracle import rocs_ref as ref
@@ -48,10 +63,8 @@ def _worker(rank, world, port, out_q):
     cfg = wl.CONFIGS[1].with_(R=7)
     co, so = wl.cand_offsets(cfg), wl.seq_offsets(cfg)
     lin, att = wl.linear_inputs(cfg, co), wl.dca_inputs(cfg, co, so)
-    cost = sharding.request_cost(np.diff(co), np.diff(so), c_attn=0.05)
-    mine = sharding.partition_requests(cost, world)[rank]
-    rows, co_l = sharding.shard_rows(co, mine)
-    seq_rows, so_l = sharding.shard_rows(so, mine)
+    sh = sharding.shard_batch(co, world, rank, seq_offsets=so, c_attn=0.05)   # the helper bench.py --gpus N uses
+    mine, rows, co_l, seq_rows, so_l = sh.requests, sh.cand_rows, sh.cand_offsets, sh.seq_rows, sh.seq_offsets
     y = ref.ikbo_linear(co_l, lin["XR"][mine], lin["XC"][rows], lin["W"])
     o = ref.dca_attention(co_l, so_l, att["Q"][rows], att["K"][seq_rows], att["V"][seq_rows])
     # timing reduction used by the benchmark: max over ranks
