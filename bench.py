@@ -235,8 +235,7 @@ def run_rocs(args):
     h1 = [torch.empty((N, 1024), dtype=torch.bfloat16, device="cuda") for _ in range(N_SETS)]
     h2 = [torch.empty((N, 1024), dtype=torch.bfloat16, device="cuda") for _ in range(N_SETS)]
     y = [torch.empty((N, 256), dtype=torch.bfloat16, device="cuda") for _ in range(N_SETS)]
-    ws_bytes = 256 * 1024 * 4
-    workspace = torch.empty(ws_bytes, dtype=torch.uint8, device="cuda")
+    workspace = torch.empty(rocs.ikbo_linear_workspace(rocs.plan_create(co_dev, co), 1024), dtype=torch.uint8, device="cuda")
     launches_per_step = 5  # fill_row2req, request half, candidate half, layer 2, layer 3
 
     def step(i, XR=None, XC=None, co_d=None, marks=None):
