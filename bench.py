@@ -498,6 +498,8 @@ def bench_other_ops(torch, rocs, peaks, dev, time_call, which):
     out = []
     if "dca" in which:
         out.append(bench_dca(torch, rocs, peaks, dev, time_call))
+    if "dh128" in which:
+        out.append(bench_dca(torch, rocs, peaks, dev, time_call, dh=128))
     if "nq" in which:
         out.append(bench_dca_nq(torch, rocs, peaks, dev, time_call, 32))
     if "nq64" in which:
@@ -599,9 +601,9 @@ def dca_record(key, name, cfg, N, co, so, t, t_fresh, t_mat, peaks, rows_per_can
     return rec
 
 
-def bench_dca(torch, rocs, peaks, dev, time_call):
-    # configuration 3: one DCA layer
-    cfg = wl.CONFIGS[3]
+def bench_dca(torch, rocs, peaks, dev, time_call, dh=64):
+    # configuration 3: one DCA layer (dh = 128: the same width as 4 heads of 128, same flops)
+    cfg = wl.CONFIGS[3] if dh == 64 else wl.CONFIGS[3].with_(H=8 * 64 // dh, dh=dh)
     co, so = wl.cand_offsets(cfg), wl.seq_offsets(cfg)
     N = int(co[-1])
     d = wl.dca_inputs(cfg, co, so)
@@ -611,6 +613,9 @@ def bench_dca(torch, rocs, peaks, dev, time_call):
     O = torch.empty_like(Q)
     t = time_call(lambda i: rocs.dca_attention(plan, Q, K, V, sod, out=O), reps=10)
     t_fresh = with_fresh_plan(rocs, time_call, co_dev, co, lambda pl: rocs.dca_attention(pl, Q, K, V, sod, out=O), reps=10)
+    if dh != 64:
+        return dca_record(f"cfg3.dca_dh{dh}", f"cfg3 dca_attention with {cfg.H} heads of {dh} (R=64, L=2048)", cfg, N, co,
+                          so, t, t_fresh, None, peaks)
     t_mat = time_call(lambda i: materialised_dca(torch, Q, K, V, co, so), reps=1, warm=1)
     return dca_record("cfg3.dca", "cfg3 dca_attention (R=64, L=2048, 8x64)", cfg, N, co, so, t, t_fresh, t_mat, peaks)
 
@@ -785,8 +790,8 @@ def main():
     ap.add_argument("--warmup", type=int, default=10)
     ap.add_argument("--impl", default="rocs", choices=["rocs", "reference"])
     ap.add_argument("--skip-extra", action="store_true", help="skip the attention / interaction side measurements")
-    ap.add_argument("--extra", default="dca,nq,nq64,glm,fm,norm,cfg5",
-                    help="side measurements to run: dca, nq, nq64, glm, fm, norm, cfg5")
+    ap.add_argument("--extra", default="dca,dh128,nq,nq64,glm,fm,norm,cfg5",
+                    help="side measurements to run: dca, dh128, nq, nq64, glm, fm, norm, cfg5")
     ap.add_argument("--skip-cpu", action="store_true", help="skip the cpu_baseline leg")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "rocs" else args.warmup

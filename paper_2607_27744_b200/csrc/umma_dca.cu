@@ -6,6 +6,9 @@
 // 128-key blocks, nothing is replicated per candidate (tiles of the same request and head are
 // consecutive items, so their K/V blocks are read from L2 at about the same time).
 //
+// Head dimensions 64 (128-key blocks) and 128 (64-key blocks: tensor memory holds S, P and O of both
+// sides in 512 columns either way); the description below gives the figures of the first.
+//
 // One persistent CTA per SM runs TWO independent item streams (sides A and B), 20 warps:
 //   warps 16,19 TMA producers of sides A, B: the Q tile of the item, then (K_j, V_j) blocks through a ring
 //   warps 17,18 tcgen05.mma issuers of sides A, B:  S = Q K_j^T (128x128x64, operands in shared memory)
@@ -39,43 +42,52 @@ namespace {
 
 using namespace ptx;
 
-constexpr int DH = 64;            // head dimension handled here (128-byte rows)
 constexpr int BQ = 128;           // query rows per tile
-constexpr int BKV = 128;          // keys per block
 constexpr int kSoftmaxWarps = 16; // 8 per side
 constexpr int kControlWarp0 = kSoftmaxWarps;   // warps 16, 19: TMA producers of sides A, B; 17, 18: their MMA issuers
 constexpr int kThreads = (kSoftmaxWarps + 4) * 32;
-constexpr int kKvStages = 3;      // per side
 constexpr int kTmemCols = 512;
-constexpr int kQBytes = BQ * DH * 2;            // 16 KB
-constexpr int kKBytes = BKV * DH * 2;           // 16 KB
-constexpr int kKvStageBytes = 2 * kKBytes;      // K block + V block
 constexpr uint32_t kStatusDca = 0x400;
 constexpr int kSideTmemStride = 256;
-constexpr int kPColOffset = 128;
-constexpr int kOColOffset = 192;
 
-// Shared-memory map (byte offsets from the 1024-byte aligned base); per side: one Q tile (freed when
-// the item's last S is issued, a block before its end) and a ring of K/V stages.
-constexpr uint32_t kOffQ = 0;                                          // [2 sides][128][64] bf16
-constexpr uint32_t kOffKv = kOffQ + 2 * kQBytes;                       // [2 sides][stages][K 16 KB | V 16 KB]
-constexpr uint32_t kOffL = kOffKv + 2 * kKvStages * kKvStageBytes;     // partial sums [2 sides][2 halves][128] fp32
-constexpr uint32_t kOffBar = kOffL + 2 * 2 * BQ * 4;
-// barriers, 8 bytes each, [side] innermost where there are two
-constexpr uint32_t kBarQFull = kOffBar;                    // [2]
-constexpr uint32_t kBarQEmpty = kBarQFull + 16;            // [2]
-constexpr uint32_t kBarKvFull = kBarQEmpty + 16;           // [2][stages]
-constexpr uint32_t kBarKvEmpty = kBarKvFull + 16 * kKvStages;
-constexpr uint32_t kBarSFull = kBarKvEmpty + 16 * kKvStages;  // [2]
-constexpr uint32_t kBarSEmpty = kBarSFull + 16;
-constexpr uint32_t kBarPFull = kBarSEmpty + 16;
-constexpr uint32_t kBarOFull = kBarPFull + 16;
-constexpr uint32_t kBarPair = kBarOFull + 16;              // [8]: the two warps that share 32 query rows
-constexpr uint32_t kBarDrain = kBarPair + 64;              // [2]
-constexpr uint32_t kOffTmemPtr = kBarDrain + 16;
-constexpr uint32_t kOffAbort = kOffTmemPtr + 4;
-constexpr int kSmemBytes = kOffAbort + 12;
-static_assert(kSmemBytes <= 232448, "shared memory of one SM");
+// Everything that depends on the head dimension DH and the keys per block BKV.  Operand tiles are kept
+// as boxes of 64 columns (128-byte rows, 128-byte swizzle): a tile of DH columns is DH / 64 boxes.
+template <int DH_, int BKV_>
+struct DcaCfg {
+  static constexpr int DH = DH_, BKV = BKV_;
+  static constexpr int kBoxes = DH / 64;
+  static constexpr int kCols = BKV / 2;                      // score columns per softmax thread
+  static constexpr int kOutCols = DH / 2;                    // output columns per softmax thread
+  static constexpr int kKvStages = DH == 64 ? 3 : 2;         // per side
+  static constexpr int kQBoxBytes = BQ * 128, kQBytes = kBoxes * kQBoxBytes;
+  static constexpr int kKvBoxBytes = BKV * 128, kKBytes = kBoxes * kKvBoxBytes;
+  static constexpr int kKvStageBytes = 2 * kKBytes;          // K block + V block
+  // tensor memory per side: S [0, BKV) fp32, P [BKV, BKV + BKV/2) bf16 pairs, O [.., + DH) fp32
+  static constexpr int kPColOffset = BKV, kOColOffset = BKV + BKV / 2;
+  static_assert(kOColOffset + DH <= kSideTmemStride, "tensor memory columns of a side");
+  static_assert(kCols == 32 || kCols == 64, "score columns per thread");
+  // Shared-memory map (byte offsets from the 1024-byte aligned base); per side: one Q tile (freed when
+  // the item's last S is issued, a block before its end) and a ring of K/V stages.
+  static constexpr uint32_t kOffQ = 0;                                          // [2 sides][boxes][128][64] bf16
+  static constexpr uint32_t kOffKv = kOffQ + 2 * kQBytes;                       // [2 sides][stages][K | V]
+  static constexpr uint32_t kOffL = kOffKv + 2 * kKvStages * kKvStageBytes;     // partial sums [2 sides][2 halves][128] fp32
+  static constexpr uint32_t kOffBar = kOffL + 2 * 2 * BQ * 4;
+  // barriers, 8 bytes each, [side] innermost where there are two
+  static constexpr uint32_t kBarQFull = kOffBar;                    // [2]
+  static constexpr uint32_t kBarQEmpty = kBarQFull + 16;            // [2]
+  static constexpr uint32_t kBarKvFull = kBarQEmpty + 16;           // [2][stages]
+  static constexpr uint32_t kBarKvEmpty = kBarKvFull + 16 * kKvStages;
+  static constexpr uint32_t kBarSFull = kBarKvEmpty + 16 * kKvStages;  // [2]
+  static constexpr uint32_t kBarSEmpty = kBarSFull + 16;
+  static constexpr uint32_t kBarPFull = kBarSEmpty + 16;
+  static constexpr uint32_t kBarOFull = kBarPFull + 16;
+  static constexpr uint32_t kBarPair = kBarOFull + 16;              // [8]: the two warps that share 32 query rows
+  static constexpr uint32_t kBarDrain = kBarPair + 64;              // [2]
+  static constexpr uint32_t kOffTmemPtr = kBarDrain + 16;
+  static constexpr uint32_t kOffAbort = kOffTmemPtr + 4;
+  static constexpr int kSmemBytes = kOffAbort + 12;
+  static_assert(kSmemBytes <= 232448, "shared memory of one SM");
+};
 
 #ifndef ROCS_DCA_EMU
 #define ROCS_DCA_EMU 0
@@ -157,11 +169,18 @@ __device__ __forceinline__ void umma_ts(uint32_t d_tmem, uint32_t a_tmem, uint64
       : "memory");
 }
 
-// One query row of one head, 32 of its 64 output columns, in plain fp32 with the row's true maximum as
-// reference: q and k point at the head's 64 values of the row / of the request's first key, v at the
-// 32 columns wanted; consecutive keys are `stride` elements apart.  Inlined on purpose: as a called
+__device__ __forceinline__ void tmem_st_32x32b_x8(uint32_t taddr, const uint32_t* r) {
+  asm volatile("tcgen05.st.sync.aligned.32x32b.x8.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8};" ::"r"(taddr), "r"(r[0]),
+               "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7])
+               : "memory");
+}
+
+// One query row of one head, half of its DH output columns, in plain fp32 with the row's true maximum
+// as reference: q and k point at the head's DH values of the row / of the request's first key, v at the
+// DH / 2 columns wanted; consecutive keys are `stride` elements apart.  Inlined on purpose: as a called
 // function it forces the caller's hot loop to keep its registers where the calling convention wants
 // them, and the loop spills.
+template <int DH>
 __device__ __forceinline__ void row_by_hand(const __nv_bfloat16* q, const __nv_bfloat16* k, const __nv_bfloat16* v,
                                             int32_t stride, int32_t L, float scale_log2e, __nv_bfloat16* out) {
   auto score = [&](int32_t j) {
@@ -171,15 +190,15 @@ __device__ __forceinline__ void row_by_hand(const __nv_bfloat16* q, const __nv_b
   };
   float m = -INFINITY;
   for (int32_t j = 0; j < L; ++j) m = fmaxf(m, score(j));
-  float acc[32], l = 0.f;
-  for (int d = 0; d < 32; ++d) acc[d] = 0.f;
+  float acc[DH / 2], l = 0.f;
+  for (int d = 0; d < DH / 2; ++d) acc[d] = 0.f;
   for (int32_t j = 0; j < L; ++j) {
     const float pj = exp2f(score(j) - m);
     l += pj;
-    for (int d = 0; d < 32; ++d) acc[d] = fmaf(pj, __bfloat162float(v[(int64_t)j * stride + d]), acc[d]);
+    for (int d = 0; d < DH / 2; ++d) acc[d] = fmaf(pj, __bfloat162float(v[(int64_t)j * stride + d]), acc[d]);
   }
   const float inv = 1.f / l;
-  for (int d = 0; d < 32; ++d) out[d] = __float2bfloat16_rn(acc[d] * inv);
+  for (int d = 0; d < DH / 2; ++d) out[d] = __float2bfloat16_rn(acc[d] * inv);
 }
 
 // A short burst of probes before the paced wait: for hand-offs that are usually complete already.
@@ -201,9 +220,19 @@ constexpr int kTraceBlocks = 96;
 #define TRACE_NEXT()
 #endif
 
+template <int DH, int BKV>
 __global__ void __launch_bounds__(kThreads, 1)
 dca_umma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
                 const __grid_constant__ CUtensorMap map_v, const DcaParams p) {
+  using C = DcaCfg<DH, BKV>;
+  constexpr int kKvStages = C::kKvStages, kBoxes = C::kBoxes, kCols = C::kCols, kOutCols = C::kOutCols;
+  constexpr int kQBytes = C::kQBytes, kKBytes = C::kKBytes, kKvStageBytes = C::kKvStageBytes;
+  constexpr int kPColOffset = C::kPColOffset, kOColOffset = C::kOColOffset;
+  constexpr uint32_t kOffQ = C::kOffQ, kOffKv = C::kOffKv, kOffL = C::kOffL, kBarQFull = C::kBarQFull,
+                     kBarQEmpty = C::kBarQEmpty, kBarKvFull = C::kBarKvFull, kBarKvEmpty = C::kBarKvEmpty,
+                     kBarSFull = C::kBarSFull, kBarSEmpty = C::kBarSEmpty, kBarPFull = C::kBarPFull,
+                     kBarOFull = C::kBarOFull, kBarPair = C::kBarPair, kBarDrain = C::kBarDrain,
+                     kOffTmemPtr = C::kOffTmemPtr, kOffAbort = C::kOffAbort;
   extern __shared__ __align__(1024) uint8_t smem[];     // swizzled operand tiles need 1024-byte alignment
   const uint32_t sb = smem_u32(smem);                   // every shared-memory address below is sb + constant
   AbortFlag* abort_flag = reinterpret_cast<AbortFlag*>(smem + kOffAbort);
@@ -263,14 +292,21 @@ dca_umma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
         if (!mbar_wait_paced(q_empty, (n_work & 1) ^ 1, abort_flag, p.status, kStatusDca | 1)) { ok = false; break; }
         ++n_work;
         mbar_expect_tx(q_full, kQBytes);
-        tma_load_2d(q_dst, &map_q, q_full, item.head * DH, item.cand0 * p.n_q);
+#pragma unroll
+        for (int bx = 0; bx < kBoxes; ++bx)
+          tma_load_2d(q_dst + bx * C::kQBoxBytes, &map_q, q_full, item.head * DH + bx * 64, item.cand0 * p.n_q);
         const int32_t nblk = (L + BKV - 1) / BKV;
         for (int32_t j = 0; j < nblk; ++j, ++kv_it) {
           const uint32_t s = kv_it % kKvStages;
           if (!mbar_wait_paced(kv_empty + 8 * s, ((kv_it / kKvStages) & 1) ^ 1, abort_flag, p.status, kStatusDca | 2)) { ok = false; break; }
           mbar_expect_tx(kv_full + 8 * s, kKvStageBytes);
-          tma_load_2d(kv_dst + s * kKvStageBytes, &map_k, kv_full + 8 * s, item.head * DH, s0 + j * BKV);
-          tma_load_2d(kv_dst + s * kKvStageBytes + kKBytes, &map_v, kv_full + 8 * s, item.head * DH, s0 + j * BKV);
+#pragma unroll
+          for (int bx = 0; bx < kBoxes; ++bx) {
+            tma_load_2d(kv_dst + s * kKvStageBytes + bx * C::kKvBoxBytes, &map_k, kv_full + 8 * s,
+                        item.head * DH + bx * 64, s0 + j * BKV);
+            tma_load_2d(kv_dst + s * kKvStageBytes + kKBytes + bx * C::kKvBoxBytes, &map_v, kv_full + 8 * s,
+                        item.head * DH + bx * 64, s0 + j * BKV);
+          }
         }
       }
       if (!ok) {
@@ -287,7 +323,7 @@ dca_umma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
     // ------------------------------ MMA issuers: one warp per side ---------------------------
     const int side = warp - (kControlWarp0 + 1);
     constexpr uint32_t idesc_s = umma_idesc_bf16(BQ, BKV, false, false);  // S = Q K^T, both K-major
-    constexpr uint32_t idesc_o = umma_idesc_bf16(BQ, DH, false, true);    // O = P V, V is MN-major
+    constexpr uint32_t idesc_o = umma_idesc_bf16(BQ, 64, false, true);    // O = P V per 64 output columns, V is MN-major
     const uint32_t q_full = sb + kBarQFull + 8 * side, q_empty = sb + kBarQEmpty + 8 * side;
     const uint32_t kv_full = sb + kBarKvFull + 8 * kKvStages * side, kv_empty = sb + kBarKvEmpty + 8 * kKvStages * side;
     const uint32_t s_full = sb + kBarSFull + 8 * side, s_empty = sb + kBarSEmpty + 8 * side;
@@ -306,7 +342,9 @@ dca_umma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
     auto desc_v = [&](uint32_t stage) { return smem_desc_sw128(kv_base + stage * kKvStageBytes + kKBytes, 1024, 16); };
     auto issue_s = [&](uint64_t b_desc) {
 #pragma unroll
-      for (int k = 0; k < DH / 16; ++k) umma_ss(t_s, dq + 2 * k, b_desc + 2 * k, idesc_s, k != 0 ? 1u : 0u);
+      for (int k = 0; k < DH / 16; ++k)  // 16 columns of dh per step: box k / 4, 32 bytes further on inside it
+        umma_ss(t_s, dq + (k / 4) * (C::kQBoxBytes >> 4) + 2 * (k % 4), b_desc + (k / 4) * (C::kKvBoxBytes >> 4) + 2 * (k % 4),
+                idesc_s, k != 0 ? 1u : 0u);
       umma_commit(s_full);
     };
     auto issue_pv = [&](uint64_t b_desc, bool first_block) {
@@ -314,8 +352,10 @@ dca_umma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
       // V: rows are keys (K), 128 bytes = 64 head dims (N): 16 keys = 2048 bytes further on
 #pragma unroll
       for (int k = 0; k < BKV / 16; ++k)
-        umma_ts(t_s + kOColOffset, t_s + kPColOffset + k * 8, b_desc + k * (16 * 128 / 16), idesc_o,
-                (k != 0 || !first_block) ? 1u : 0u);
+#pragma unroll
+        for (int bx = 0; bx < kBoxes; ++bx)  // 64 output columns per product
+          umma_ts(t_s + kOColOffset + bx * 64, t_s + kPColOffset + k * 8,
+                  b_desc + bx * (C::kKvBoxBytes >> 4) + k * (16 * 128 / 16), idesc_o, (k != 0 || !first_block) ? 1u : 0u);
       umma_commit(o_full);
     };
     // The last block of a sequence may reach past it into the next request's rows (or past the
@@ -324,8 +364,9 @@ dca_umma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
     // request) cannot reach this request's output.
     auto zero_v_tail = [&](uint32_t stage, int32_t valid) {
       uint8_t* v = smem + kOffKv + (side * kKvStages + stage) * kKvStageBytes + kKBytes;
-      for (int idx = valid * 8 + lane; idx < BKV * 8; idx += 32)
-        *reinterpret_cast<uint4*>(v + idx * 16) = make_uint4(0u, 0u, 0u, 0u);
+      for (int bx = 0; bx < kBoxes; ++bx)
+        for (int idx = valid * 8 + lane; idx < BKV * 8; idx += 32)
+          *reinterpret_cast<uint4*>(v + bx * C::kKvBoxBytes + idx * 16) = make_uint4(0u, 0u, 0u, 0u);
       fence_proxy_async_smem();
       __syncwarp();
     };
@@ -391,13 +432,13 @@ dca_umma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
   } else {
     // ------------------------------ softmax warps ------------------------------------------
     const int side = warp >> 3;
-    const int half = (warp >> 2) & 1;       // which 64 of the block's 128 key columns
+    const int half = (warp >> 2) & 1;       // which half of the block's key columns
     const int q = warp & 3;                 // TMEM lane quadrant this warp may touch
     const int row = q * 32 + lane;          // query row of the tile = TMEM lane
     const uint32_t t_row = tmem_base + side * kSideTmemStride + ((uint32_t)(q * 32) << 16);  // S columns of the row
-    const uint32_t t_s = t_row + half * 64;
-    const uint32_t t_p = t_row + kPColOffset + half * 32;
-    const uint32_t t_o = t_row + kOColOffset + half * 32;
+    const uint32_t t_s = t_row + half * kCols;
+    const uint32_t t_p = t_row + kPColOffset + half * (kCols / 2);
+    const uint32_t t_o = t_row + kOColOffset + half * kOutCols;
     const uint32_t s_full = sb + kBarSFull + 8 * side, s_empty = sb + kBarSEmpty + 8 * side;
     const uint32_t p_full = sb + kBarPFull + 8 * side, o_full = sb + kBarOFull + 8 * side;
     const uint32_t my_pair = sb + kBarPair + 8 * (side * 4 + q);
@@ -413,8 +454,8 @@ dca_umma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
       const DcaItem item = p.items[i];
       const int32_t L = p.seq_offsets[item.req + 1] - p.seq_offsets[item.req];
       const int32_t rows_valid = item.count_a * p.n_q;
-      // this thread's 32 output columns of its row
-      auto out_ptr = [&]() { return p.O + ((int64_t)item.cand0 * p.n_q + row) * row_width + item.head * DH + half * 32; };
+      // this thread's half of the output columns of its row
+      auto out_ptr = [&]() { return p.O + ((int64_t)item.cand0 * p.n_q + row) * row_width + item.head * DH + half * kOutCols; };
       bool aborted = false;
       if (L > 0) {
         const int32_t nblk = (L + BKV - 1) / BKV;
@@ -458,21 +499,24 @@ dca_umma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
           }
           ++cnt_s;
           TRACE_SM(1);
-          uint32_t sv[64];  // this thread's 64 scores of the block
-          tmem_ld_32x32b_x32(t_s, sv);
-          tmem_ld_32x32b_x32(t_s + 32, sv + 32);
+          uint32_t sv[kCols];  // this thread's scores of the block
+#pragma unroll
+          for (int c = 0; c < kCols; c += 32) tmem_ld_32x32b_x32(t_s + c, sv + c);
           tmem_ld_wait();
           tc_fence_before_sync();
           __syncwarp();
           if (lane == 0) mbar_arrive(s_empty);  // S_{j+1} may overwrite the tile now
-          const int32_t valid = L - j * BKV - half * 64;  // columns of this thread's half that are keys of the request
-          if (valid < 64) {
+          const int32_t valid = L - j * BKV - half * kCols;  // columns of this thread's half that are keys of the request
+          if (valid < kCols) {
 #pragma unroll
-            for (int e = 0; e < 64; ++e)
+            for (int e = 0; e < kCols; ++e)
               if (e >= valid) sv[e] = 0xff800000u;  // -inf: the key does not exist
           }
           TRACE_SM(2);
-          uint32_t pk[16];  // P of 32 keys of this row, bf16 pairs; stored in two halves
+          uint32_t pk[kCols / 4];  // P of half of this thread's keys, bf16 pairs; stored in two halves
+          auto store_p = [&](uint32_t taddr) {
+            if constexpr (kCols == 64) tmem_st_32x32b_x16(taddr, pk); else tmem_st_32x32b_x8(taddr, pk);
+          };
           auto exp_pair = [&](int e) {
             float p0, p1;
             if (((e >> 1) & 7) < kEmuPairs) {
@@ -498,10 +542,10 @@ dca_umma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
               p1 = ex2(x1);
             }
             sum2 = fadd2(sum2, pack2(p0, p1));
-            pk[(e / 2) & 15] = bf16x2_bits(p0, p1);
+            pk[(e / 2) % (kCols / 4)] = bf16x2_bits(p0, p1);
           };
 #pragma unroll
-          for (int e = 0; e < 32; e += 2) exp_pair(e);
+          for (int e = 0; e < kCols / 2; e += 2) exp_pair(e);
           TRACE_SM(3);
           if (j > 0) {
             // P V of the previous block has read P_{j-1} (it was issued most of a block ago): from here
@@ -511,11 +555,11 @@ dca_umma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
           }
           ++cnt_o;
           TRACE_SM(4);
-          tmem_st_32x32b_x16(t_p, pk);
+          store_p(t_p);
 #pragma unroll
-          for (int e = 32; e < 64; e += 2) exp_pair(e);
+          for (int e = kCols / 2; e < kCols; e += 2) exp_pair(e);
           TRACE_SM(5);
-          tmem_st_32x32b_x16(t_p + 16, pk);
+          store_p(t_p + kCols / 4);
           if (kEmuPairs > 0 && g_max * p.scale_log2e - m_ref > 126.f) by_hand = true;  // 2^n would leave fp32's exponent field
           tmem_st_wait();
           tc_fence_before_sync();
@@ -540,19 +584,20 @@ dca_umma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
         const float l_o = l_x[(side * 2 + (half ^ 1)) * BQ + row];
         const float l_tot = half == 0 ? l_run + l_o : l_o + l_run;  // same order in both halves
         const float inv = 1.f / l_tot;
-        uint32_t v[32];
-        tmem_ld_32x32b_x32(t_o, v);
+        uint32_t v[kOutCols];
+#pragma unroll
+        for (int c = 0; c < kOutCols; c += 32) tmem_ld_32x32b_x32(t_o + c, v + c);
         tmem_ld_wait();
         // Scores that outgrow the first block's maximum by 2^128 or so overflow fp32 (and so can
         // a sum of products with huge values): the row then holds Inf or NaN instead of a result.
         float probe = l_tot * 0.f;
 #pragma unroll
-        for (int e = 0; e < 32; ++e) probe = fmaf(__uint_as_float(v[e]), 0.f, probe);
+        for (int e = 0; e < kOutCols; ++e) probe = fmaf(__uint_as_float(v[e]), 0.f, probe);
         if (row < rows_valid) {
           __nv_bfloat16* out = out_ptr();
           if (probe == 0.f && !by_hand) {
 #pragma unroll
-            for (int e = 0; e < 32; e += 8) {
+            for (int e = 0; e < kOutCols; e += 8) {
               uint4 w;
               w.x = bf16x2_bits(__uint_as_float(v[e + 0]) * inv, __uint_as_float(v[e + 1]) * inv);
               w.y = bf16x2_bits(__uint_as_float(v[e + 2]) * inv, __uint_as_float(v[e + 3]) * inv);
@@ -564,15 +609,15 @@ dca_umma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
             // such a row is computed again here, by this thread alone, with its true maximum as reference
             const int64_t q_row = (int64_t)item.cand0 * p.n_q + row;
             const int64_t kv0 = ((int64_t)p.seq_offsets[item.req] * p.H + item.head) * DH;
-            row_by_hand(p.Q + q_row * row_width + item.head * DH, p.K + kv0, p.V + kv0 + half * 32, row_width, L,
-                        p.scale_log2e, out);
+            row_by_hand<DH>(p.Q + q_row * row_width + item.head * DH, p.K + kv0, p.V + kv0 + half * kOutCols, row_width,
+                            L, p.scale_log2e, out);
           }
         }
       } else if (row < rows_valid) {
         // a request without keys: zero rows
         __nv_bfloat16* out = out_ptr();
 #pragma unroll
-        for (int c = 0; c < 32; c += 8) *reinterpret_cast<uint4*>(out + c) = make_uint4(0u, 0u, 0u, 0u);
+        for (int c = 0; c < kOutCols; c += 8) *reinterpret_cast<uint4*>(out + c) = make_uint4(0u, 0u, 0u, 0u);
       }
       tc_fence_before_sync();  // the next item's first P V overwrites O
     }
@@ -599,26 +644,26 @@ int sm_count_dca() {
 }  // namespace
 
 bool umma_dca_supported(int32_t n_q, int32_t H, int32_t dh) {
-  return dh == DH && n_q >= 1 && n_q <= BQ && H >= 1 && H <= 65535;
+  return (dh == 64 || dh == 128) && n_q >= 1 && n_q <= BQ && H >= 1 && H <= 65535;
 }
 
-rocs_status_t umma_dca(const rocs_plan* plan, int32_t n_q, int32_t H, int32_t dh, float scale, const void* Q,
-                       const void* K, const void* V, const int32_t* seq_offsets, int64_t T, void* O,
-                       cudaStream_t stream) {
-  (void)dh;
-  if (plan->N == 0) return ROCS_OK;
+template <int DH, int BKV>
+static rocs_status_t launch_dca(const rocs_plan* plan, int32_t n_q, int32_t H, float scale, const void* Q,
+                                const void* K, const void* V, const int32_t* seq_offsets, int64_t T, void* O,
+                                cudaStream_t stream) {
+  using C = DcaCfg<DH, BKV>;
   DcaItemList items;
   rocs_status_t st = plan_dca_items(plan, BQ / n_q, H, /*tiles_per_item=*/1, stream, &items);
   if (st != ROCS_OK) return st;
   if (items.num == 0) return ROCS_OK;
   const uint64_t width = (uint64_t)H * DH;
   CUtensorMap map_q, map_k, map_v;
-  if (!make_tensor_map_2d(&map_q, Q, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, (uint64_t)plan->N * n_q, width, width, BQ, DH,
+  if (!make_tensor_map_2d(&map_q, Q, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, (uint64_t)plan->N * n_q, width, width, BQ, 64,
                           true))
     return ROCS_ERR_CUDA;
   if (T > 0) {
-    if (!make_tensor_map_2d(&map_k, K, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, (uint64_t)T, width, width, BKV, DH, true) ||
-        !make_tensor_map_2d(&map_v, V, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, (uint64_t)T, width, width, BKV, DH, true))
+    if (!make_tensor_map_2d(&map_k, K, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, (uint64_t)T, width, width, BKV, 64, true) ||
+        !make_tensor_map_2d(&map_v, V, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, (uint64_t)T, width, width, BKV, 64, true))
       return ROCS_ERR_CUDA;
   } else {
     map_k = map_q;  // every sequence is empty: the kernel only writes zeros
@@ -641,11 +686,20 @@ rocs_status_t umma_dca(const rocs_plan* plan, int32_t n_q, int32_t H, int32_t dh
 #ifdef ROCS_DCA_TRACE
   p.trace = (long long*)rocs_dca_trace_buffer;
 #endif
-  ROCS_CUDA_TRY(cudaFuncSetAttribute(dca_umma_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes));
+  auto kernel = dca_umma_kernel<DH, BKV>;
+  ROCS_CUDA_TRY(cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, C::kSmemBytes));
   const int grid = std::min((items.num + 1) / 2, sm_count_dca());  // one CTA per SM, two item streams per CTA
-  dca_umma_kernel<<<grid, kThreads, kSmemBytes, stream>>>(map_q, map_k, map_v, p);
+  kernel<<<grid, kThreads, C::kSmemBytes, stream>>>(map_q, map_k, map_v, p);
   ROCS_CUDA_TRY(cudaGetLastError());
   return ROCS_OK;
+}
+
+rocs_status_t umma_dca(const rocs_plan* plan, int32_t n_q, int32_t H, int32_t dh, float scale, const void* Q,
+                       const void* K, const void* V, const int32_t* seq_offsets, int64_t T, void* O,
+                       cudaStream_t stream) {
+  if (plan->N == 0) return ROCS_OK;
+  if (dh == 64) return launch_dca<64, 128>(plan, n_q, H, scale, Q, K, V, seq_offsets, T, O, stream);
+  return launch_dca<128, 64>(plan, n_q, H, scale, Q, K, V, seq_offsets, T, O, stream);
 }
 
 }  // namespace rocs
