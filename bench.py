@@ -461,7 +461,8 @@ def run_rocs(args):
         out = {"us": round(l["us"], 1)}
         for k_in, k_out in (("frac", "frac"), ("frac_hbm", "frac_hbm"), ("frac_tensor", "frac_tensor_burst"),
                             ("frac_of_exp_unit_peak_at_max_clock", "frac_exp_unit"),
-                            ("speedup_vs_materialised", "x_materialised"), ("us_with_fresh_plan", "us_fresh_plan")):
+                            ("speedup_vs_materialised", "x_materialised"), ("us_with_fresh_plan", "us_fresh_plan"),
+                            ("unfused_us", "unfused_us")):
             if k_in in l and l[k_in] is not None:
                 out[k_out] = round(l[k_in], 3 if "frac" in k_out else 1)
         return out
@@ -510,6 +511,8 @@ def bench_other_ops(torch, rocs, peaks, dev, time_call, which):
         out.append(bench_fm(torch, rocs, peaks, dev, time_call))
     if "norm" in which:
         out.append(bench_norm(torch, rocs, peaks, dev, time_call))
+    if "normfused" in which:
+        out.append(bench_norm_fused(torch, rocs, peaks, dev, time_call))
     if "cfg5" in which:
         out.extend(bench_cfg5(torch, rocs, peaks, dev, time_call))
     return out
@@ -721,6 +724,40 @@ def bench_norm(torch, rocs, peaks, dev, time_call):
             "note": "input and output (537 MB) are larger than L2"}
 
 
+def bench_norm_fused(torch, rocs, peaks, dev, time_call):
+    """Configuration 2 with an RMSNorm between layers 1 and 2 (Eq. 7): folded into the two layers (layer 1
+    leaves the row sums, layer 2 scales its accumulators) against layer 1, the stand-alone normalisation
+    kernel and layer 2."""
+    cfg = wl.CONFIGS[2]
+    co = wl.cand_offsets(cfg)
+    N = int(co[-1])
+    lin, ws = wl.linear_inputs(cfg, co), wl.mlp_weights(cfg)
+    co_dev = dev(co)
+    plan = rocs.plan_create(co_dev, co)
+    XR, XC, W1, W2 = dev(lin["XR"]), dev(lin["XC"]), dev(lin["W"]), dev(ws[0])
+    W1_cr, W1_cc = W1[:, :cfg.d_req], W1[:, cfg.d_req:]
+    gamma = torch.ones(cfg.d_out, dtype=torch.bfloat16, device="cuda")
+    h1 = torch.empty((N, cfg.d_out), dtype=torch.bfloat16, device="cuda")
+    hn = torch.empty_like(h1)
+    h2 = torch.empty((N, 1024), dtype=torch.bfloat16, device="cuda")
+    stats = torch.empty((N, 2), dtype=torch.float32, device="cuda")
+    wsp = torch.empty(int(rocs.lib().rocs_ikbo_linear_stats_workspace(plan.handle, cfg.d_out)), dtype=torch.uint8, device="cuda")
+
+    def fused(i):
+        rocs.ikbo_linear_stats(plan, XR, XC, W1_cr, W1_cc, relu=True, out=h1, row_stats=stats, workspace=wsp)
+        rocs.linear_normed(h1, stats, W2, None, None, 1e-6, rocs.NORM_RMS, relu=True, out=h2)
+
+    def unfused(i):
+        rocs.ikbo_linear(plan, XR, XC, W1_cr, W1_cc, relu=True, out=h1, workspace=wsp)
+        rocs.group_norm(h1, gamma, None, 1e-6, rocs.NORM_RMS, out=hn)
+        rocs.linear(hn, W2, relu=True, out=h2)
+
+    t_f, t_u = time_call(fused, reps=20), time_call(unfused, reps=20)
+    return {"key": "cfg2.norm_fused", "layer": "cfg2 layers 1-2 with an RMSNorm between them, folded into both layers",
+            "N": N, "us": t_f * 1e6, "cand_per_s": N / t_f, "unfused_us": t_u * 1e6, "speedup_vs_unfused": t_u / t_f,
+            "note": "unfused = split layer, stand-alone group-norm kernel (reads and writes the 268 MB activation), plain layer"}
+
+
 def bench_cfg5(torch, rocs, peaks, dev, time_call):
     """Configuration 5 (skewed, Zipf candidate counts): the three calls timed independently, each
     against a materialised-broadcast GPU path."""
@@ -790,8 +827,8 @@ def main():
     ap.add_argument("--warmup", type=int, default=10)
     ap.add_argument("--impl", default="rocs", choices=["rocs", "reference"])
     ap.add_argument("--skip-extra", action="store_true", help="skip the attention / interaction side measurements")
-    ap.add_argument("--extra", default="dca,dh128,nq,nq64,glm,fm,norm,cfg5",
-                    help="side measurements to run: dca, dh128, nq, nq64, glm, fm, norm, cfg5")
+    ap.add_argument("--extra", default="dca,dh128,nq,nq64,glm,fm,norm,normfused,cfg5",
+                    help="side measurements to run: dca, dh128, nq, nq64, glm, fm, norm, normfused, cfg5")
     ap.add_argument("--skip-cpu", action="store_true", help="skip the cpu_baseline leg")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "rocs" else args.warmup

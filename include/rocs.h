@@ -248,6 +248,43 @@ rocs_status_t rocs_group_norm(rocs_dtype_t dtype, rocs_norm_t kind, int64_t M, i
                               int64_t ld_y, void* stream);
 
 /*
+ * Group-local normalisation folded into the layers around it (Eq. 7 together with the fused
+ * epilogue of Section 4.2.1): for a row y and the layer that consumes norm(y),
+ *     LayerNorm:  norm(y) W^T = sc (y W^T) + sh (W 1),   sc = 1 / sqrt(var(y) + eps), sh = -mean(y) sc
+ *     RMSNorm:    norm(y) W^T = sc (y W^T),              sc = 1 / sqrt(mean(y^2) + eps)
+ * so the normalised rows are never written: the layer that produces y leaves each row's sum and
+ * sum of squares (rocs_ikbo_linear_stats), the layer that consumes it scales and shifts its own
+ * accumulators (rocs_linear_normed).  A learned gain gamma and offset beta are folded by the caller:
+ * pass W with its columns multiplied by gamma and bias + W beta.
+ *
+ * rocs_ikbo_linear_stats: rocs_ikbo_linear plus
+ *   row_stats [N, 2] fp32   (sum, sum of squares) over the d_out outputs of each row (after the
+ *                           activation; taken from the fp32 values before they are rounded)
+ *   workspace               >= rocs_ikbo_linear_stats_workspace(plan, d_out) bytes, 256-byte aligned
+ * rocs_weight_row_sums: wbar[n] = sum_k W[n, k] in fp32 (the W 1 of LayerNorm's shift).
+ * rocs_linear_normed: Y = act(norm(X) W^T + bias) from X as stored, its row_stats [M, 2] and wbar
+ *   (wbar may be NULL for ROCS_NORM_RMS).  The variance is taken as mean(x^2) - mean(x)^2 in fp32:
+ *   rows whose mean is thousands of times their spread lose accuracy; rocs_group_norm has no such limit.
+ *   bf16 rows on the wide-layer kernel only (M >= 2048, d_out >= 256 and a multiple of 8); other
+ *   shapes return ROCS_ERR_UNSUPPORTED: normalise with rocs_group_norm, then call rocs_linear.
+ * Errors: INVALID_ARG, ALIGNMENT, WORKSPACE, UNSUPPORTED, CUDA.
+ */
+size_t rocs_ikbo_linear_stats_workspace(const rocs_plan_t* plan, int32_t d_out);
+rocs_status_t rocs_ikbo_linear_stats(const rocs_plan_t* plan, rocs_dtype_t dtype, int32_t d_req,
+                                     int32_t d_cand, int32_t d_out, const void* XR, int64_t ld_xr,
+                                     const void* XC, int64_t ld_xc, const void* W_CR, int64_t ld_wcr,
+                                     const void* W_CC, int64_t ld_wcc, const float* bias,
+                                     rocs_act_t act, void* Y, int64_t ld_y, float* row_stats,
+                                     void* workspace, size_t workspace_bytes, void* stream);
+rocs_status_t rocs_weight_row_sums(rocs_dtype_t dtype, int32_t d_out, int32_t d_in, const void* W,
+                                   int64_t ld_w, float* wbar, void* stream);
+rocs_status_t rocs_linear_normed(rocs_dtype_t dtype, rocs_norm_t kind, int64_t M, int32_t d_in,
+                                 int32_t d_out, const void* X, int64_t ld_x, const float* row_stats,
+                                 float eps, const void* W, int64_t ld_w, const float* wbar,
+                                 const float* bias, rocs_act_t act, void* Y, int64_t ld_y,
+                                 void* stream);
+
+/*
  * Device-side status of the tensor-core kernels.  Their barrier waits are bounded; a wait
  * that expires records a code in a device word instead of spinning forever and the kernel
  * returns.  This call synchronises the device, reads the word, clears it and returns

@@ -32,7 +32,8 @@ EXPORTS = [
     "rocs_dca_attention", "rocs_glm_interaction_workspace", "rocs_glm_interaction",
     "rocs_glm_fm_projection_workspace", "rocs_glm_fm_projection", "rocs_group_norm",
     "rocs_last_device_status", "rocs_ikbo_linear_static", "rocs_ikbo_linear_static_max_z_elems",
-    "rocs_ikbo_linear_static_max_candidates",
+    "rocs_ikbo_linear_static_max_candidates", "rocs_ikbo_linear_stats_workspace", "rocs_ikbo_linear_stats",
+    "rocs_weight_row_sums", "rocs_linear_normed",
 ]
 
 
@@ -76,6 +77,13 @@ def lib() -> ctypes.CDLL:
         L.rocs_glm_fm_projection.argtypes = [vp, ctypes.c_int, i32, i32, i32, i32, vp, vp, vp, vp, vp, vp, sz, vp]
         L.rocs_group_norm.argtypes = [ctypes.c_int, ctypes.c_int, i64, i32, vp, i64, vp, vp, f32, vp, i64, vp]
         L.rocs_last_device_status.argtypes = [ctypes.POINTER(ctypes.c_uint32)]
+        L.rocs_ikbo_linear_stats_workspace.restype = sz
+        L.rocs_ikbo_linear_stats_workspace.argtypes = [vp, i32]
+        L.rocs_ikbo_linear_stats.argtypes = [vp, ctypes.c_int, i32, i32, i32, vp, i64, vp, i64, vp, i64, vp, i64,
+                                             vp, ctypes.c_int, vp, i64, vp, vp, sz, vp]
+        L.rocs_weight_row_sums.argtypes = [ctypes.c_int, i32, i32, vp, i64, vp, vp]
+        L.rocs_linear_normed.argtypes = [ctypes.c_int, ctypes.c_int, i64, i32, i32, vp, i64, vp, f32, vp, i64, vp, vp,
+                                         ctypes.c_int, vp, i64, vp]
         L.rocs_ikbo_linear_static_max_z_elems.restype = sz
         L.rocs_ikbo_linear_static_max_candidates.restype = sz
         L.rocs_ikbo_linear_static.argtypes = [ctypes.c_int, i32, i64, vp, i32, i32, i32, vp, i64, vp, i64, vp, i64,
@@ -191,6 +199,55 @@ def ikbo_linear(plan: Plan, XR: Optional[torch.Tensor], XC: torch.Tensor, W_CR: 
         _p(bias), ACT_RELU if relu else ACT_NONE, _p(out), _rows_2d(out),
         _p(workspace), workspace.numel() if workspace is not None else 0, _stream())
     _check(code, "rocs_ikbo_linear")
+    return out
+
+
+def ikbo_linear_stats(plan: Plan, XR: torch.Tensor, XC: torch.Tensor, W_CR: torch.Tensor, W_CC: torch.Tensor,
+                      bias: Optional[torch.Tensor] = None, relu: bool = False, out: Optional[torch.Tensor] = None,
+                      row_stats: Optional[torch.Tensor] = None, workspace: Optional[torch.Tensor] = None):
+    """ikbo_linear that also leaves each output row's (sum, sum of squares) for a normalisation folded
+    into the next layer (Eq. 7).  Returns (Y, row_stats [N, 2] fp32)."""
+    d_req, d_cand, d_out = XR.shape[1], XC.shape[1], W_CC.shape[0]
+    assert XC.shape[0] == plan.N
+    if out is None:
+        out = torch.empty((plan.N, d_out), dtype=XC.dtype, device=XC.device)
+    if row_stats is None:
+        row_stats = torch.empty((plan.N, 2), dtype=torch.float32, device=XC.device)
+    need = int(lib().rocs_ikbo_linear_stats_workspace(plan.handle, d_out))
+    if workspace is None:
+        workspace = torch.empty(need, dtype=torch.uint8, device=XC.device)
+    code = lib().rocs_ikbo_linear_stats(
+        plan.handle, _dtype_code(XC), d_req, d_cand, d_out, _p(XR), _rows_2d(XR), _p(XC), _rows_2d(XC),
+        _p(W_CR), _rows_2d(W_CR), _p(W_CC), _rows_2d(W_CC), _p(bias), ACT_RELU if relu else ACT_NONE, _p(out),
+        _rows_2d(out), _p(row_stats), _p(workspace), workspace.numel(), _stream())
+    _check(code, "rocs_ikbo_linear_stats")
+    return out, row_stats
+
+
+def weight_row_sums(W: torch.Tensor, out: Optional[torch.Tensor] = None) -> torch.Tensor:
+    """wbar[n] = sum_k W[n, k] in fp32: the W 1 term of a LayerNorm folded into the layer."""
+    d_out, d_in = W.shape
+    if out is None:
+        out = torch.empty(d_out, dtype=torch.float32, device=W.device)
+    _check(lib().rocs_weight_row_sums(_dtype_code(W), d_out, d_in, _p(W), _rows_2d(W), _p(out), _stream()),
+           "rocs_weight_row_sums")
+    return out
+
+
+def linear_normed(X: torch.Tensor, row_stats: torch.Tensor, W: torch.Tensor, wbar: Optional[torch.Tensor] = None,
+                  bias: Optional[torch.Tensor] = None, eps: float = 1e-5, kind: int = NORM_LAYER, relu: bool = False,
+                  out: Optional[torch.Tensor] = None) -> torch.Tensor:
+    """Y = act(norm(X) W^T + bias) with the normalisation applied to the layer's accumulators (Eq. 7
+    folded into the epilogue); gamma and beta are folded into W and bias by the caller."""
+    M, d_in = X.shape
+    d_out = W.shape[0]
+    assert row_stats.dtype == torch.float32 and row_stats.shape == (M, 2) and row_stats.is_contiguous()
+    if out is None:
+        out = torch.empty((M, d_out), dtype=X.dtype, device=X.device)
+    code = lib().rocs_linear_normed(_dtype_code(X), kind, M, d_in, d_out, _p(X), _rows_2d(X), _p(row_stats), float(eps),
+                                    _p(W), _rows_2d(W), _p(wbar), _p(bias), ACT_RELU if relu else ACT_NONE, _p(out),
+                                    _rows_2d(out), _stream())
+    _check(code, "rocs_linear_normed")
     return out
 
 

@@ -290,21 +290,23 @@ static rocs_status_t linear_dispatch(rocs_dtype_t dt, int64_t M, int32_t d_in, i
                                      const float* bias, const float* add, int64_t ld_add,
                                      const int32_t* row2req, int act, void* Y, int64_t ld_y,
                                      bool out_f32, cudaStream_t stream,
-                                     bool add_from_previous_launch = false) {
+                                     bool add_from_previous_launch = false, float2* stat_partials = nullptr) {
   if (dt == ROCS_BF16 && g_path.load() == ROCS_PATH_AUTO &&
       umma_linear_supported(M, d_in, d_out, ld_x, ld_w, ld_y, out_f32))
     return umma_linear(M, d_in, d_out, X, ld_x, W, ld_w, bias, add, ld_add, row2req, act, Y, ld_y,
-                       out_f32, stream, add_from_previous_launch);
+                       out_f32, stream, add_from_previous_launch, stat_partials);
   return simt_linear(dt, M, d_in, d_out, X, ld_x, W, ld_w, bias, add, ld_add, row2req, act, Y, ld_y,
                      out_f32, stream);
 }
 
-rocs_status_t rocs_ikbo_linear(const rocs_plan_t* plan, rocs_dtype_t dtype, int32_t d_req,
-                               int32_t d_cand, int32_t d_out, const void* XR, int64_t ld_xr,
-                               const void* XC, int64_t ld_xc, const void* W_CR, int64_t ld_wcr,
-                               const void* W_CC, int64_t ld_wcc, const float* bias, rocs_act_t act,
-                               void* Y, int64_t ld_y, void* workspace, size_t workspace_bytes,
-                               void* stream_) {
+// row_stats (optional): per-row (sum, sum of squares) of the output, for a normalisation folded into
+// the next layer; its partials follow Z in the workspace.
+static rocs_status_t ikbo_linear_impl(const rocs_plan_t* plan, rocs_dtype_t dtype, int32_t d_req,
+                                      int32_t d_cand, int32_t d_out, const void* XR, int64_t ld_xr,
+                                      const void* XC, int64_t ld_xc, const void* W_CR, int64_t ld_wcr,
+                                      const void* W_CC, int64_t ld_wcc, const float* bias, rocs_act_t act,
+                                      void* Y, int64_t ld_y, float* row_stats, void* workspace,
+                                      size_t workspace_bytes, void* stream_) {
   if (!plan || (dtype != ROCS_BF16 && dtype != ROCS_F32)) return ROCS_ERR_INVALID_ARG;
   if (d_req < 0 || d_cand < 0 || d_out <= 0 || d_req + d_cand <= 0) return ROCS_ERR_INVALID_ARG;
   if (act != ROCS_ACT_NONE && act != ROCS_ACT_RELU) return ROCS_ERR_INVALID_ARG;
@@ -320,8 +322,15 @@ rocs_status_t rocs_ikbo_linear(const rocs_plan_t* plan, rocs_dtype_t dtype, int3
     return ROCS_ERR_ALIGNMENT;
   cudaStream_t stream = (cudaStream_t)stream_;
   const float* Z = nullptr;
+  const size_t z_bytes = d_req > 0 ? rocs_ikbo_linear_workspace(plan, d_out) : 0;
+  if (row_stats != nullptr) {
+    if (!aligned16(row_stats) || d_cand <= 0) return row_stats && d_cand <= 0 ? ROCS_ERR_INVALID_ARG : ROCS_ERR_ALIGNMENT;
+    const size_t need = rocs_ikbo_linear_stats_workspace(plan, d_out);
+    if (!workspace || workspace_bytes < need || (reinterpret_cast<uintptr_t>(workspace) & 255u))
+      return ROCS_ERR_WORKSPACE;
+  }
   if (d_req > 0) {
-    const size_t need = rocs_ikbo_linear_workspace(plan, d_out);
+    const size_t need = z_bytes;
     if (!workspace || workspace_bytes < need || (reinterpret_cast<uintptr_t>(workspace) & 255u))
       return ROCS_ERR_WORKSPACE;
     // Request half, once per request (Section 4.1): Z = X^R W_CR^T + bias, fp32.
@@ -337,9 +346,80 @@ rocs_status_t rocs_ikbo_linear(const rocs_plan_t* plan, rocs_dtype_t dtype, int3
   // with it (it waits for it before reading Z).  Only meaningful when both went to tensor cores.
   const bool request_half_on_umma = Z != nullptr && dtype == ROCS_BF16 && g_path.load() == ROCS_PATH_AUTO &&
                                     umma_linear_supported(plan->R, d_req, d_out, ld_xr, ld_wcr, d_out, true);
-  return linear_dispatch(dtype, plan->N, d_cand, d_out, XC, ld_xc, W_CC, ld_wcc, bias, Z, d_out,
-                         Z ? plan->row2req : nullptr, act, Y, ld_y, /*out_f32=*/false, stream,
-                         request_half_on_umma);
+  // Row sums for a following normalisation: left as partials by the candidate kernel's epilogue where
+  // the CTA-pair kernel runs (and added up by a small kernel), otherwise taken from the stored output.
+  float2* partials = nullptr;
+  if (row_stats != nullptr && dtype == ROCS_BF16 && g_path.load() == ROCS_PATH_AUTO &&
+      umma_linear_supported(plan->N, d_cand, d_out, ld_xc, ld_wcc, ld_y, false) &&
+      umma_linear_ws2_supported(plan->N, d_cand, d_out, false))
+    partials = reinterpret_cast<float2*>(static_cast<uint8_t*>(workspace) + z_bytes);
+  rocs_status_t st = linear_dispatch(dtype, plan->N, d_cand, d_out, XC, ld_xc, W_CC, ld_wcc, bias, Z, d_out,
+                                     Z ? plan->row2req : nullptr, act, Y, ld_y, /*out_f32=*/false, stream,
+                                     request_half_on_umma, partials);
+  if (st != ROCS_OK || row_stats == nullptr) return st;
+  if (partials != nullptr)
+    return row_stats_from_partials(plan->N, umma_linear_ws2_stat_partials(d_out), partials,
+                                   reinterpret_cast<float2*>(row_stats), stream);
+  return row_stats_direct(dtype, plan->N, d_out, Y, ld_y, reinterpret_cast<float2*>(row_stats), stream);
+}
+
+rocs_status_t rocs_ikbo_linear(const rocs_plan_t* plan, rocs_dtype_t dtype, int32_t d_req,
+                               int32_t d_cand, int32_t d_out, const void* XR, int64_t ld_xr,
+                               const void* XC, int64_t ld_xc, const void* W_CR, int64_t ld_wcr,
+                               const void* W_CC, int64_t ld_wcc, const float* bias, rocs_act_t act,
+                               void* Y, int64_t ld_y, void* workspace, size_t workspace_bytes,
+                               void* stream_) {
+  return ikbo_linear_impl(plan, dtype, d_req, d_cand, d_out, XR, ld_xr, XC, ld_xc, W_CR, ld_wcr, W_CC, ld_wcc, bias,
+                          act, Y, ld_y, nullptr, workspace, workspace_bytes, stream_);
+}
+
+size_t rocs_ikbo_linear_stats_workspace(const rocs_plan_t* plan, int32_t d_out) {
+  if (!plan || d_out <= 0) return 0;
+  return rocs_ikbo_linear_workspace(plan, d_out) +
+         round_up((size_t)plan->N * (size_t)umma_linear_ws2_stat_partials(d_out) * sizeof(float2), 256);
+}
+
+rocs_status_t rocs_ikbo_linear_stats(const rocs_plan_t* plan, rocs_dtype_t dtype, int32_t d_req,
+                                     int32_t d_cand, int32_t d_out, const void* XR, int64_t ld_xr,
+                                     const void* XC, int64_t ld_xc, const void* W_CR, int64_t ld_wcr,
+                                     const void* W_CC, int64_t ld_wcc, const float* bias, rocs_act_t act,
+                                     void* Y, int64_t ld_y, float* row_stats, void* workspace,
+                                     size_t workspace_bytes, void* stream_) {
+  if (!row_stats && plan && plan->N > 0) return ROCS_ERR_INVALID_ARG;
+  return ikbo_linear_impl(plan, dtype, d_req, d_cand, d_out, XR, ld_xr, XC, ld_xc, W_CR, ld_wcr, W_CC, ld_wcc, bias,
+                          act, Y, ld_y, row_stats, workspace, workspace_bytes, stream_);
+}
+
+rocs_status_t rocs_weight_row_sums(rocs_dtype_t dtype, int32_t d_out, int32_t d_in, const void* W, int64_t ld_w,
+                                   float* wbar, void* stream_) {
+  if ((dtype != ROCS_BF16 && dtype != ROCS_F32) || d_out <= 0 || d_in <= 0 || !W || !wbar) return ROCS_ERR_INVALID_ARG;
+  if (!aligned16(W) || !aligned16(wbar) || !row_stride_ok(ld_w, d_in, dtype)) return ROCS_ERR_ALIGNMENT;
+  return weight_row_sums(dtype, d_out, d_in, W, ld_w, wbar, (cudaStream_t)stream_);
+}
+
+rocs_status_t rocs_linear_normed(rocs_dtype_t dtype, rocs_norm_t kind, int64_t M, int32_t d_in, int32_t d_out,
+                                 const void* X, int64_t ld_x, const float* row_stats, float eps, const void* W,
+                                 int64_t ld_w, const float* wbar, const float* bias, rocs_act_t act, void* Y,
+                                 int64_t ld_y, void* stream_) {
+  if ((dtype != ROCS_BF16 && dtype != ROCS_F32) || (kind != ROCS_NORM_LAYER && kind != ROCS_NORM_RMS))
+    return ROCS_ERR_INVALID_ARG;
+  if (M < 0 || d_in <= 0 || d_out <= 0 || !X || !W || !Y || !row_stats || !(eps >= 0.f)) return ROCS_ERR_INVALID_ARG;
+  if (kind == ROCS_NORM_LAYER && !wbar) return ROCS_ERR_INVALID_ARG;
+  if (act != ROCS_ACT_NONE && act != ROCS_ACT_RELU) return ROCS_ERR_INVALID_ARG;
+  if (!aligned16(X) || !aligned16(W) || !aligned16(Y) || !aligned16(bias) || !aligned16(wbar) || !aligned16(row_stats) ||
+      !row_stride_ok(ld_x, d_in, dtype) || !row_stride_ok(ld_w, d_in, dtype) || !row_stride_ok(ld_y, d_out, dtype))
+    return ROCS_ERR_ALIGNMENT;
+  // The folded form lives in the epilogue of the wide-layer kernel; other shapes normalise with
+  // rocs_group_norm and call rocs_linear.
+  if (dtype != ROCS_BF16 || g_path.load() != ROCS_PATH_AUTO || d_out % 4 != 0 ||
+      !umma_linear_pair_supported(M, d_in, d_out, false, false))
+    return ROCS_ERR_UNSUPPORTED;
+  RowNorm norm;
+  norm.row_stats = reinterpret_cast<const float2*>(row_stats);
+  norm.kind = (int)kind;
+  norm.eps = eps;
+  norm.wbar = wbar;
+  return umma_linear_pair(M, d_in, d_out, X, ld_x, W, ld_w, bias, (int)act, Y, ld_y, (cudaStream_t)stream_, &norm);
 }
 
 rocs_status_t rocs_linear(rocs_dtype_t dtype, int64_t M, int32_t d_in, int32_t d_out, const void* X,

@@ -113,19 +113,39 @@ bool umma_linear_supported(int64_t M, int32_t d_in, int32_t d_out, int64_t ld_x,
 rocs_status_t umma_linear(int64_t M, int32_t d_in, int32_t d_out, const void* X, int64_t ld_x,
                           const void* W, int64_t ld_w, const float* bias, const float* add,
                           int64_t ld_add, const int32_t* row2req, int act, void* Y, int64_t ld_y,
-                          bool out_f32, cudaStream_t stream, bool add_from_previous_launch = false);
+                          bool out_f32, cudaStream_t stream, bool add_from_previous_launch = false,
+                          float2* stat_partials = nullptr);
 // Weight-stationary kernel on CTA pairs (cta_group::2) for d_in <= 256 and bf16 output: half a weight
 // slice per SM, TMA-store epilogue (umma_linear picks it when it applies).
 bool umma_linear_ws2_supported(int64_t M, int32_t d_in, int32_t d_out, bool out_f32);
 rocs_status_t umma_linear_ws2(int64_t M, int32_t d_in, int32_t d_out, const void* X, int64_t ld_x,
                               const void* W, int64_t ld_w, const float* bias, const float* add,
                               int64_t ld_add, const int32_t* row2req, int act, void* Y, int64_t ld_y,
-                              cudaStream_t stream, bool add_from_previous_launch = false);
+                              cudaStream_t stream, bool add_from_previous_launch = false,
+                              float2* stat_partials = nullptr);
+// Number of (sum, sum of squares) partials per row the kernel above writes when asked to.
+inline int32_t umma_linear_ws2_stat_partials(int32_t d_out) { return 2 * ((d_out + 255) / 256); }
 // K-ring GEMM on CTA pairs for wide plain layers (no request term, bf16 output, many rows).
 bool umma_linear_pair_supported(int64_t M, int32_t d_in, int32_t d_out, bool out_f32, bool has_add);
+// norm (optional): the rows of X are to be normalised (Eq. 7) before the product; the kernel applies the
+// row's scale and shift to its accumulators instead (see rocs_linear_normed).
+struct RowNorm {
+  const float2* row_stats = nullptr;  // [M] (sum, sum of squares) over the d_in columns of each row of X
+  int kind = 0;                       // ROCS_NORM_LAYER / ROCS_NORM_RMS
+  float eps = 0.f;
+  const float* wbar = nullptr;        // [d_out] row sums of W (LayerNorm only)
+};
 rocs_status_t umma_linear_pair(int64_t M, int32_t d_in, int32_t d_out, const void* X, int64_t ld_x,
                                const void* W, int64_t ld_w, const float* bias, int act, void* Y,
-                               int64_t ld_y, cudaStream_t stream);
+                               int64_t ld_y, cudaStream_t stream, const RowNorm* norm = nullptr);
+
+// ---- per-row sums for a normalisation fused into the next layer: row_stats.cu ---------------------
+rocs_status_t row_stats_from_partials(int64_t M, int32_t partials_per_row, const float2* partials, float2* row_stats,
+                                      cudaStream_t stream);
+rocs_status_t row_stats_direct(rocs_dtype_t dt, int64_t M, int32_t d, const void* Y, int64_t ld_y, float2* row_stats,
+                               cudaStream_t stream);
+rocs_status_t weight_row_sums(rocs_dtype_t dt, int32_t d_out, int32_t d_in, const void* W, int64_t ld_w, float* wbar,
+                              cudaStream_t stream);
 bool umma_dca_supported(int32_t n_q, int32_t H, int32_t dh);
 rocs_status_t umma_dca(const rocs_plan* plan, int32_t n_q, int32_t H, int32_t dh, float scale,
                        const void* Q, const void* K, const void* V, const int32_t* seq_offsets,

@@ -36,6 +36,13 @@ struct PairParams {
   const float* bias;
   int32_t act;
   uint32_t* status;
+  // optional normalisation of the input rows, folded into the epilogue:
+  //   norm(x) W^T = sc (x W^T) + sh wbar,  sc = 1 / sqrt(var + eps), sh = -mean sc   (LayerNorm)
+  //                                        sc = 1 / sqrt(mean(x^2) + eps), sh = 0    (RMSNorm)
+  const float2* in_stats;   // [M] (sum, sum of squares) of each input row, or NULL
+  const float* wbar;        // [d_out] row sums of W (LayerNorm)
+  int32_t norm_kind;
+  float eps, inv_d;
 };
 
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kThreads, 1)
@@ -155,6 +162,18 @@ linear_pair_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_const
       if (lane == 0) tma_store_wait_read<0>();  // the previous tile's stores have read this warp's boxes
       __syncwarp();
       const uint32_t t_row = tmem_base + acc * BN + half * 128 + ((uint32_t)(q * 32) << 16);
+      float sc = 1.f, sh = 0.f;
+      if (p.in_stats != nullptr) {
+        const int64_t row = (int64_t)m0 + q * 32 + lane;
+        const float2 st = row < p.M ? __ldg(&p.in_stats[row]) : make_float2(0.f, 0.f);
+        const float mean = st.x * p.inv_d, ms = st.y * p.inv_d;
+        if (p.norm_kind == ROCS_NORM_RMS) {
+          sc = rsqrtf(ms + p.eps);
+        } else {
+          sc = rsqrtf(fmaxf(ms - mean * mean, 0.f) + p.eps);
+          sh = -mean * sc;
+        }
+      }
 #pragma unroll
       for (int c = 0; c < 2; ++c) {
         const int32_t col0 = n0 + half * 128 + c * 64;
@@ -170,6 +189,20 @@ linear_pair_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_const
         float f[64];
 #pragma unroll
         for (int i = 0; i < 64; ++i) f[i] = __uint_as_float(v[i]);
+        if (p.in_stats != nullptr) {
+#pragma unroll
+          for (int i = 0; i < 64; ++i) f[i] *= sc;
+          if (p.norm_kind != ROCS_NORM_RMS) {
+#pragma unroll
+            for (int i = 0; i < 64; i += 4) {
+              if (col0 + i < p.d_out) {
+                const float4 w = __ldg(reinterpret_cast<const float4*>(p.wbar + col0 + i));
+                f[i] = fmaf(sh, w.x, f[i]); f[i + 1] = fmaf(sh, w.y, f[i + 1]);
+                f[i + 2] = fmaf(sh, w.z, f[i + 2]); f[i + 3] = fmaf(sh, w.w, f[i + 3]);
+              }
+            }
+          }
+        }
         if (p.bias != nullptr) {
 #pragma unroll
           for (int i = 0; i < 64; i += 4) {
@@ -239,7 +272,8 @@ bool umma_linear_pair_supported(int64_t M, int32_t d_in, int32_t d_out, bool out
 }
 
 rocs_status_t umma_linear_pair(int64_t M, int32_t d_in, int32_t d_out, const void* X, int64_t ld_x, const void* W,
-                               int64_t ld_w, const float* bias, int act, void* Y, int64_t ld_y, cudaStream_t stream) {
+                               int64_t ld_w, const float* bias, int act, void* Y, int64_t ld_y, cudaStream_t stream,
+                               const RowNorm* norm) {
   CUtensorMap map_x, map_w, map_y;
   if (!make_tensor_map_2d(&map_x, X, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, (uint64_t)M, (uint64_t)d_in, (uint64_t)ld_x,
                           BM, BK, true) ||
@@ -250,7 +284,14 @@ rocs_status_t umma_linear_pair(int64_t M, int32_t d_in, int32_t d_out, const voi
     return ROCS_ERR_CUDA;
   uint32_t* status = device_status_word();
   if (!status) return ROCS_ERR_CUDA;
-  PairParams p{M, d_in, d_out, bias, act, status};
+  PairParams p{M, d_in, d_out, bias, act, status, nullptr, nullptr, 0, 0.f, 0.f};
+  if (norm != nullptr) {
+    p.in_stats = norm->row_stats;
+    p.wbar = norm->wbar;
+    p.norm_kind = norm->kind;
+    p.eps = norm->eps;
+    p.inv_d = 1.f / (float)d_in;
+  }
   const int64_t tiles = ((M + 2 * BM - 1) / (2 * BM)) * ((d_out + BN - 1) / BN);
   const int pairs = (int)std::min<int64_t>(tiles, sm_count_pair() / 2);
   ROCS_CUDA_TRY(cudaFuncSetAttribute(linear_pair_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes));

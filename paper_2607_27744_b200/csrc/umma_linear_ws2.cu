@@ -51,6 +51,7 @@ struct Ws2Params {
   const int32_t* row2req;
   int32_t act;
   int32_t wait_for_previous;  // launched with programmatic serialization behind the kernel that writes `add`
+  float2* stat_partials;      // [M][2 n_slices] (sum, sum of squares) of each row's 128 columns per epilogue warp, or NULL
   uint32_t* status;
 };
 
@@ -228,6 +229,7 @@ linear_ws2_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_consta
       if (lane == 0) tma_store_wait_read<0>();
       __syncwarp();
       const uint32_t t_row = tmem_base + acc * BN + half * 128 + ((uint32_t)(q * 32) << 16);
+      float st_sum = 0.f, st_sq = 0.f;  // this row's 128 output columns, for a normalisation that follows (Eq. 7)
 #pragma unroll
       for (int c = 0; c < 2; ++c) {
         const int32_t colL = half * 128 + c * 64;   // column inside the slice
@@ -273,6 +275,13 @@ linear_ws2_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_consta
 #pragma unroll
           for (int i = 0; i < 64; ++i) f[i] = fmaxf(f[i], 0.f);
         }
+        if (p.stat_partials != nullptr) {  // columns past d_out hold zeros and add nothing
+#pragma unroll
+          for (int i = 0; i < 64; ++i) {
+            st_sum += f[i];
+            st_sq = fmaf(f[i], f[i], st_sq);
+          }
+        }
         if (c == 1) {  // the store of the first chunk has finished reading the box
           if (lane == 0) tma_store_wait_read<0>();
           __syncwarp();
@@ -299,6 +308,8 @@ linear_ws2_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_consta
           tma_store_commit();
         }
       }
+      if (p.stat_partials != nullptr && row < p.M)
+        p.stat_partials[row * (2 * p.n_slices) + slice * 2 + half] = make_float2(st_sum, st_sq);
       if (lane == 0 && has_add) mbar_arrive(&z_empty[lt % kZBufs]);
     }
     if (lane == 0) tma_store_wait_all<0>();
@@ -333,7 +344,7 @@ bool umma_linear_ws2_supported(int64_t M, int32_t d_in, int32_t d_out, bool out_
 rocs_status_t umma_linear_ws2(int64_t M, int32_t d_in, int32_t d_out, const void* X, int64_t ld_x, const void* W,
                               int64_t ld_w, const float* bias, const float* add, int64_t ld_add,
                               const int32_t* row2req, int act, void* Y, int64_t ld_y, cudaStream_t stream,
-                              bool add_from_previous_launch) {
+                              bool add_from_previous_launch, float2* stat_partials) {
   const int32_t k_blocks = (d_in + BK - 1) / BK;
   CUtensorMap map_x, map_w, map_z, map_y;
   if (!make_tensor_map_2d(&map_x, X, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, (uint64_t)M, (uint64_t)d_in, (uint64_t)ld_x,
@@ -361,6 +372,7 @@ rocs_status_t umma_linear_ws2(int64_t M, int32_t d_in, int32_t d_out, const void
   p.a_stages = std::min(10, (227 * 1024 - fixed) / kAStageBytes);
   p.bias = bias; p.add = add; p.ld_add = ld_add; p.row2req = row2req; p.act = act; p.status = status;
   p.wait_for_previous = (add_from_previous_launch && add != nullptr) ? 1 : 0;
+  p.stat_partials = stat_partials;
   const int smem_bytes = fixed + p.a_stages * kAStageBytes;
   ROCS_CUDA_TRY(cudaFuncSetAttribute(linear_ws2_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_bytes));
   cudaLaunchConfig_t cfg = {};
