@@ -290,11 +290,12 @@ static rocs_status_t linear_dispatch(rocs_dtype_t dt, int64_t M, int32_t d_in, i
                                      const float* bias, const float* add, int64_t ld_add,
                                      const int32_t* row2req, int act, void* Y, int64_t ld_y,
                                      bool out_f32, cudaStream_t stream,
-                                     bool add_from_previous_launch = false, float2* stat_partials = nullptr) {
+                                     bool add_from_previous_launch = false, float2* stat_partials = nullptr,
+                                     int64_t add_rows = 0) {
   if (dt == ROCS_BF16 && g_path.load() == ROCS_PATH_AUTO &&
       umma_linear_supported(M, d_in, d_out, ld_x, ld_w, ld_y, out_f32))
     return umma_linear(M, d_in, d_out, X, ld_x, W, ld_w, bias, add, ld_add, row2req, act, Y, ld_y,
-                       out_f32, stream, add_from_previous_launch, stat_partials);
+                       out_f32, stream, add_from_previous_launch, stat_partials, add_rows);
   return simt_linear(dt, M, d_in, d_out, X, ld_x, W, ld_w, bias, add, ld_add, row2req, act, Y, ld_y,
                      out_f32, stream);
 }
@@ -355,7 +356,7 @@ static rocs_status_t ikbo_linear_impl(const rocs_plan_t* plan, rocs_dtype_t dtyp
     partials = reinterpret_cast<float2*>(static_cast<uint8_t*>(workspace) + z_bytes);
   rocs_status_t st = linear_dispatch(dtype, plan->N, d_cand, d_out, XC, ld_xc, W_CC, ld_wcc, bias, Z, d_out,
                                      Z ? plan->row2req : nullptr, act, Y, ld_y, /*out_f32=*/false, stream,
-                                     request_half_on_umma, partials);
+                                     request_half_on_umma, partials, plan->R);
   if (st != ROCS_OK || row_stats == nullptr) return st;
   if (partials != nullptr)
     return row_stats_from_partials(plan->N, umma_linear_ws2_stat_partials(d_out), partials,

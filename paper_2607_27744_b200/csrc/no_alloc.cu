@@ -59,10 +59,10 @@ bool stride_ok(int64_t ld, int64_t cols, rocs_dtype_t dt) {
 rocs_status_t run_linear(rocs_dtype_t dt, int64_t M, int32_t d_in, int32_t d_out, const void* X, int64_t ld_x,
                          const void* W, int64_t ld_w, const float* bias, const float* add, int64_t ld_add,
                          const int32_t* row2req, int act, void* Y, int64_t ld_y, bool out_f32,
-                         cudaStream_t stream) {
+                         cudaStream_t stream, int64_t add_rows = 0) {
   if (dt == ROCS_BF16 && umma_linear_supported(M, d_in, d_out, ld_x, ld_w, ld_y, out_f32))
     return umma_linear(M, d_in, d_out, X, ld_x, W, ld_w, bias, add, ld_add, row2req, act, Y, ld_y, out_f32,
-                       stream);
+                       stream, false, nullptr, add_rows);
   return simt_linear(dt, M, d_in, d_out, X, ld_x, W, ld_w, bias, add, ld_add, row2req, act, Y, ld_y, out_f32,
                      stream);
 }
@@ -107,7 +107,7 @@ rocs_status_t rocs_ikbo_linear_static(rocs_dtype_t dtype, int32_t R, int64_t N, 
                   d_out, /*out_f32=*/true, stream);
   if (st != ROCS_OK) return st;
   return run_linear(dtype, N, d_cand, d_out, XC, ld_xc, W_CC, ld_wcc, nullptr, Z, d_out, map, act, Y, ld_y,
-                    /*out_f32=*/false, stream);
+                    /*out_f32=*/false, stream, R);
 }
 
 }  // extern "C"

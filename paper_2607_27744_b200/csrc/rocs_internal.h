@@ -107,6 +107,7 @@ rocs_status_t fm_projection(rocs_dtype_t dt, const rocs_plan* plan, int32_t n_r,
 // ---- tcgen05 tensor-core kernels (bf16): umma_*.cu -------------------------------------
 bool umma_linear_supported(int64_t M, int32_t d_in, int32_t d_out, int64_t ld_x, int64_t ld_w,
                            int64_t ld_y, bool out_f32);
+// add_rows: number of rows of `add` (the requests of the batch); 0 means one row per output row.
 // add_from_previous_launch: `add` is written by the launch directly in front of this one on the
 // stream (the request half) and nothing else this call reads is; the kernel may then overlap its
 // set-up with that launch and waits for it only before it reads `add`.
@@ -114,7 +115,7 @@ rocs_status_t umma_linear(int64_t M, int32_t d_in, int32_t d_out, const void* X,
                           const void* W, int64_t ld_w, const float* bias, const float* add,
                           int64_t ld_add, const int32_t* row2req, int act, void* Y, int64_t ld_y,
                           bool out_f32, cudaStream_t stream, bool add_from_previous_launch = false,
-                          float2* stat_partials = nullptr);
+                          float2* stat_partials = nullptr, int64_t add_rows = 0);
 // Weight-stationary kernel on CTA pairs (cta_group::2) for d_in <= 256 and bf16 output: half a weight
 // slice per SM, TMA-store epilogue (umma_linear picks it when it applies).
 bool umma_linear_ws2_supported(int64_t M, int32_t d_in, int32_t d_out, bool out_f32);
@@ -122,7 +123,7 @@ rocs_status_t umma_linear_ws2(int64_t M, int32_t d_in, int32_t d_out, const void
                               const void* W, int64_t ld_w, const float* bias, const float* add,
                               int64_t ld_add, const int32_t* row2req, int act, void* Y, int64_t ld_y,
                               cudaStream_t stream, bool add_from_previous_launch = false,
-                              float2* stat_partials = nullptr);
+                              float2* stat_partials = nullptr, int64_t add_rows = 0);
 // Number of (sum, sum of squares) partials per row the kernel above writes when asked to.
 inline int32_t umma_linear_ws2_stat_partials(int32_t d_out) { return 2 * ((d_out + 255) / 256); }
 // K-ring GEMM on CTA pairs for wide plain layers (no request term, bf16 output, many rows).

@@ -314,10 +314,11 @@ bool umma_linear_supported(int64_t M, int32_t d_in, int32_t d_out, int64_t ld_x,
 rocs_status_t umma_linear(int64_t M, int32_t d_in, int32_t d_out, const void* X, int64_t ld_x, const void* W,
                           int64_t ld_w, const float* bias, const float* add, int64_t ld_add,
                           const int32_t* row2req, int act, void* Y, int64_t ld_y, bool out_f32,
-                          cudaStream_t stream, bool add_from_previous_launch, float2* stat_partials) {
+                          cudaStream_t stream, bool add_from_previous_launch, float2* stat_partials,
+                          int64_t add_rows) {
   if (umma_linear_ws2_supported(M, d_in, d_out, out_f32))
     return umma_linear_ws2(M, d_in, d_out, X, ld_x, W, ld_w, bias, add, ld_add, row2req, act, Y, ld_y, stream,
-                           add_from_previous_launch, stat_partials);
+                           add_from_previous_launch, stat_partials, add_rows);
   if (stat_partials != nullptr) return ROCS_ERR_UNSUPPORTED;  // the caller asks for them only where the kernel above applies
   if (umma_linear_pair_supported(M, d_in, d_out, out_f32, add != nullptr))
     return umma_linear_pair(M, d_in, d_out, X, ld_x, W, ld_w, bias, act, Y, ld_y, stream);

@@ -344,7 +344,7 @@ bool umma_linear_ws2_supported(int64_t M, int32_t d_in, int32_t d_out, bool out_
 rocs_status_t umma_linear_ws2(int64_t M, int32_t d_in, int32_t d_out, const void* X, int64_t ld_x, const void* W,
                               int64_t ld_w, const float* bias, const float* add, int64_t ld_add,
                               const int32_t* row2req, int act, void* Y, int64_t ld_y, cudaStream_t stream,
-                              bool add_from_previous_launch, float2* stat_partials) {
+                              bool add_from_previous_launch, float2* stat_partials, int64_t add_rows) {
   const int32_t k_blocks = (d_in + BK - 1) / BK;
   CUtensorMap map_x, map_w, map_z, map_y;
   if (!make_tensor_map_2d(&map_x, X, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, (uint64_t)M, (uint64_t)d_in, (uint64_t)ld_x,
@@ -355,7 +355,8 @@ rocs_status_t umma_linear_ws2(int64_t M, int32_t d_in, int32_t d_out, const void
                           32, 64, true))
     return ROCS_ERR_CUDA;
   if (add != nullptr) {
-    if (!make_tensor_map_2d(&map_z, add, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, (uint64_t)0x7fffffff, (uint64_t)d_out,
+    const int64_t z_rows = add_rows > 0 ? add_rows : M;   // a row past the last request reads as zero fill
+    if (!make_tensor_map_2d(&map_z, add, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, (uint64_t)z_rows, (uint64_t)d_out,
                             (uint64_t)ld_add, 1, BN, false))
       return ROCS_ERR_CUDA;
   } else {
