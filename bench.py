@@ -517,6 +517,8 @@ def bench_other_ops(torch, rocs, peaks, dev, time_call, which):
         out.append(bench_dca(torch, rocs, peaks, dev, time_call))
     if "dh128" in which:
         out.append(bench_dca(torch, rocs, peaks, dev, time_call, dh=128))
+    if "dh32" in which:
+        out.append(bench_dca(torch, rocs, peaks, dev, time_call, dh=32))
     if "nq" in which:
         out.append(bench_dca_nq(torch, rocs, peaks, dev, time_call, 32))
     if "nq64" in which:
@@ -621,7 +623,7 @@ def dca_record(key, name, cfg, N, co, so, t, t_fresh, t_mat, peaks, rows_per_can
 
 
 def bench_dca(torch, rocs, peaks, dev, time_call, dh=64):
-    # configuration 3: one DCA layer (dh = 128: the same width as 4 heads of 128, same flops)
+    # configuration 3: one DCA layer (dh = 128 / 32: the same width as 4 heads of 128 / 16 of 32, same flops)
     cfg = wl.CONFIGS[3] if dh == 64 else wl.CONFIGS[3].with_(H=8 * 64 // dh, dh=dh)
     co, so = wl.cand_offsets(cfg), wl.seq_offsets(cfg)
     N = int(co[-1])
@@ -843,8 +845,8 @@ def main():
     ap.add_argument("--warmup", type=int, default=10)
     ap.add_argument("--impl", default="rocs", choices=["rocs", "reference"])
     ap.add_argument("--skip-extra", action="store_true", help="skip the attention / interaction side measurements")
-    ap.add_argument("--extra", default="dca,dh128,nq,nq64,glm,fm,norm,normfused,cfg5",
-                    help="side measurements to run: dca, dh128, nq, nq64, glm, fm, norm, normfused, cfg5")
+    ap.add_argument("--extra", default="dca,dh128,dh32,nq,nq64,glm,fm,norm,normfused,cfg5",
+                    help="side measurements to run: dca, dh128, dh32, nq, nq64, glm, fm, norm, normfused, cfg5")
     ap.add_argument("--skip-cpu", action="store_true", help="skip the cpu_baseline leg")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "rocs" else args.warmup

@@ -188,6 +188,18 @@ __device__ __forceinline__ uint64_t smem_desc_sw128(uint32_t smem_addr, uint32_t
   return d;
 }
 
+// The same with 64-byte rows (32 bf16) and the 64-byte swizzle: 16-byte chunks XOR-ed with
+// (row / 2) % 4, 8-row groups 512 bytes apart; the tile base must be 512-byte aligned.
+__device__ __forceinline__ uint64_t smem_desc_sw64(uint32_t smem_addr, uint32_t sbo_bytes, uint32_t lbo_bytes) {
+  uint64_t d = 0;
+  d |= static_cast<uint64_t>((smem_addr & 0x3FFFFu) >> 4);
+  d |= static_cast<uint64_t>((lbo_bytes >> 4) & 0x3FFFu) << 16;
+  d |= static_cast<uint64_t>((sbo_bytes >> 4) & 0x3FFFu) << 32;
+  d |= static_cast<uint64_t>(1) << 46;  // descriptor version of sm_100
+  d |= static_cast<uint64_t>(4) << 61;  // 64-byte swizzle
+  return d;
+}
+
 // tcgen05.mma instruction descriptor, kind::f16: bf16 A and B, fp32 accumulator.
 // a_mn_major / b_mn_major: operand stored with its M (or N) index contiguous instead of K.
 __host__ __device__ constexpr uint32_t umma_idesc_bf16(uint32_t M, uint32_t N, bool a_mn_major, bool b_mn_major) {
@@ -354,9 +366,9 @@ __device__ __forceinline__ void umma_commit_pair(uint64_t* bar, uint16_t cta_mas
 
 // ---- host side: tensor maps through the driver entry point (no link-time libcuda) -------------
 // rows x cols row-major tensor with `ld` elements between rows; box = box_rows x box_cols.
-// swizzle128: box_cols * elem_bytes must be 128.  Returns false on failure.
+// swizzle128: box_cols * elem_bytes must be 128; swizzle64 (takes precedence): 64.  Returns false on failure.
 bool make_tensor_map_2d(CUtensorMap* map, const void* base, CUtensorMapDataType dtype, uint32_t elem_bytes,
                         uint64_t rows, uint64_t cols, uint64_t ld, uint32_t box_rows, uint32_t box_cols,
-                        bool swizzle128);
+                        bool swizzle128, bool swizzle64 = false);
 
 }  // namespace rocs

@@ -6,8 +6,9 @@
 // 128-key blocks, nothing is replicated per candidate (tiles of the same request and head are
 // consecutive items, so their K/V blocks are read from L2 at about the same time).
 //
-// Head dimensions 64 (128-key blocks) and 128 (64-key blocks: tensor memory holds S, P and O of both
-// sides in 512 columns either way); the description below gives the figures of the first.
+// Head dimensions 64 (128-key blocks), 128 (64-key blocks: tensor memory holds S, P and O of both
+// sides in 512 columns either way) and 32 (128-key blocks, operand rows of 64 bytes under the 64-byte
+// swizzle); the description below gives the figures of the first.
 //
 // One persistent CTA per SM runs TWO independent item streams (sides A and B), 20 warps:
 //   warps 16,19 TMA producers of sides A, B: the Q tile of the item, then (K_j, V_j) blocks through a ring
@@ -51,16 +52,24 @@ constexpr uint32_t kStatusDca = 0x400;
 constexpr int kSideTmemStride = 256;
 
 // Everything that depends on the head dimension DH and the keys per block BKV.  Operand tiles are kept
-// as boxes of 64 columns (128-byte rows, 128-byte swizzle): a tile of DH columns is DH / 64 boxes.
+// as boxes of 64 columns (128-byte rows, 128-byte swizzle): a tile of DH columns is DH / 64 boxes; a head
+// dimension of 32 is one box of 32 columns (64-byte rows, 64-byte swizzle).
 template <int DH_, int BKV_>
 struct DcaCfg {
   static constexpr int DH = DH_, BKV = BKV_;
-  static constexpr int kBoxes = DH / 64;
+  static constexpr int kBoxCols = DH < 64 ? DH : 64;         // columns of a box = output columns per P V product
+  static constexpr int kRowBytes = kBoxCols * 2;             // 128 or 64: also the swizzle span
+  static constexpr int kBoxes = DH / kBoxCols;
+  static_assert(kRowBytes == 128 || kRowBytes == 64, "operand rows");
   static constexpr int kCols = BKV / 2;                      // score columns per softmax thread
   static constexpr int kOutCols = DH / 2;                    // output columns per softmax thread
-  static constexpr int kKvStages = DH == 64 ? 3 : 2;         // per side
-  static constexpr int kQBoxBytes = BQ * 128, kQBytes = kBoxes * kQBoxBytes;
-  static constexpr int kKvBoxBytes = BKV * 128, kKBytes = kBoxes * kKvBoxBytes;
+  static constexpr int kKvStages = DH == 128 ? 2 : DH == 64 ? 3 : 4;  // per side
+  static constexpr int kQBoxBytes = BQ * kRowBytes, kQBytes = kBoxes * kQBoxBytes;
+  static constexpr int kKvBoxBytes = BKV * kRowBytes, kKBytes = kBoxes * kKvBoxBytes;
+  // operand descriptor of a tile of 8-row groups, rows of kRowBytes
+  __device__ static uint64_t desc(uint32_t addr) {
+    return kRowBytes == 128 ? smem_desc_sw128(addr, 1024, 16) : smem_desc_sw64(addr, 512, 16);
+  }
   static constexpr int kKvStageBytes = 2 * kKBytes;          // K block + V block
   // tensor memory per side: S [0, BKV) fp32, P [BKV, BKV + BKV/2) bf16 pairs, O [.., + DH) fp32
   static constexpr int kPColOffset = BKV, kOColOffset = BKV + BKV / 2;
@@ -294,7 +303,7 @@ dca_umma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
         mbar_expect_tx(q_full, kQBytes);
 #pragma unroll
         for (int bx = 0; bx < kBoxes; ++bx)
-          tma_load_2d(q_dst + bx * C::kQBoxBytes, &map_q, q_full, item.head * DH + bx * 64, item.cand0 * p.n_q);
+          tma_load_2d(q_dst + bx * C::kQBoxBytes, &map_q, q_full, item.head * DH + bx * C::kBoxCols, item.cand0 * p.n_q);
         const int32_t nblk = (L + BKV - 1) / BKV;
         for (int32_t j = 0; j < nblk; ++j, ++kv_it) {
           const uint32_t s = kv_it % kKvStages;
@@ -303,9 +312,9 @@ dca_umma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
 #pragma unroll
           for (int bx = 0; bx < kBoxes; ++bx) {
             tma_load_2d(kv_dst + s * kKvStageBytes + bx * C::kKvBoxBytes, &map_k, kv_full + 8 * s,
-                        item.head * DH + bx * 64, s0 + j * BKV);
+                        item.head * DH + bx * C::kBoxCols, s0 + j * BKV);
             tma_load_2d(kv_dst + s * kKvStageBytes + kKBytes + bx * C::kKvBoxBytes, &map_v, kv_full + 8 * s,
-                        item.head * DH + bx * 64, s0 + j * BKV);
+                        item.head * DH + bx * C::kBoxCols, s0 + j * BKV);
           }
         }
       }
@@ -323,7 +332,7 @@ dca_umma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
     // ------------------------------ MMA issuers: one warp per side ---------------------------
     const int side = warp - (kControlWarp0 + 1);
     constexpr uint32_t idesc_s = umma_idesc_bf16(BQ, BKV, false, false);  // S = Q K^T, both K-major
-    constexpr uint32_t idesc_o = umma_idesc_bf16(BQ, 64, false, true);    // O = P V per 64 output columns, V is MN-major
+    constexpr uint32_t idesc_o = umma_idesc_bf16(BQ, C::kBoxCols, false, true);  // O = P V per box of output columns, V is MN-major
     const uint32_t q_full = sb + kBarQFull + 8 * side, q_empty = sb + kBarQEmpty + 8 * side;
     const uint32_t kv_full = sb + kBarKvFull + 8 * kKvStages * side, kv_empty = sb + kBarKvEmpty + 8 * kKvStages * side;
     const uint32_t s_full = sb + kBarSFull + 8 * side, s_empty = sb + kBarSEmpty + 8 * side;
@@ -337,25 +346,27 @@ dca_umma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
 #endif
     const uint32_t t_s = tmem_base + side * kSideTmemStride;
     // Q tile of this side, K block and V block of a stage as shared-memory operand descriptors
-    const uint64_t dq = smem_desc_sw128(sb + kOffQ + side * kQBytes, 1024, 16);
-    auto desc_k = [&](uint32_t stage) { return smem_desc_sw128(kv_base + stage * kKvStageBytes, 1024, 16); };
-    auto desc_v = [&](uint32_t stage) { return smem_desc_sw128(kv_base + stage * kKvStageBytes + kKBytes, 1024, 16); };
+    const uint64_t dq = C::desc(sb + kOffQ + side * kQBytes);
+    auto desc_k = [&](uint32_t stage) { return C::desc(kv_base + stage * kKvStageBytes); };
+    auto desc_v = [&](uint32_t stage) { return C::desc(kv_base + stage * kKvStageBytes + kKBytes); };
     auto issue_s = [&](uint64_t b_desc) {
 #pragma unroll
-      for (int k = 0; k < DH / 16; ++k)  // 16 columns of dh per step: box k / 4, 32 bytes further on inside it
-        umma_ss(t_s, dq + (k / 4) * (C::kQBoxBytes >> 4) + 2 * (k % 4), b_desc + (k / 4) * (C::kKvBoxBytes >> 4) + 2 * (k % 4),
-                idesc_s, k != 0 ? 1u : 0u);
+      for (int k = 0; k < DH / 16; ++k) {  // 16 columns of dh per step: box k / kPerBox, 32 bytes further on inside it
+        constexpr int kPerBox = C::kBoxCols / 16;
+        umma_ss(t_s, dq + (k / kPerBox) * (C::kQBoxBytes >> 4) + 2 * (k % kPerBox),
+                b_desc + (k / kPerBox) * (C::kKvBoxBytes >> 4) + 2 * (k % kPerBox), idesc_s, k != 0 ? 1u : 0u);
+      }
       umma_commit(s_full);
     };
     auto issue_pv = [&](uint64_t b_desc, bool first_block) {
       // P: 16 keys = 8 columns of bf16 pairs in tensor memory
-      // V: rows are keys (K), 128 bytes = 64 head dims (N): 16 keys = 2048 bytes further on
+      // V: rows are keys (K), one row = a box of head dims (N): 16 keys = 16 rows further on
 #pragma unroll
       for (int k = 0; k < BKV / 16; ++k)
 #pragma unroll
-        for (int bx = 0; bx < kBoxes; ++bx)  // 64 output columns per product
-          umma_ts(t_s + kOColOffset + bx * 64, t_s + kPColOffset + k * 8,
-                  b_desc + bx * (C::kKvBoxBytes >> 4) + k * (16 * 128 / 16), idesc_o, (k != 0 || !first_block) ? 1u : 0u);
+        for (int bx = 0; bx < kBoxes; ++bx)  // one box of output columns per product
+          umma_ts(t_s + kOColOffset + bx * C::kBoxCols, t_s + kPColOffset + k * 8,
+                  b_desc + bx * (C::kKvBoxBytes >> 4) + k * (16 * C::kRowBytes / 16), idesc_o, (k != 0 || !first_block) ? 1u : 0u);
       umma_commit(o_full);
     };
     // The last block of a sequence may reach past it into the next request's rows (or past the
@@ -365,7 +376,7 @@ dca_umma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
     auto zero_v_tail = [&](uint32_t stage, int32_t valid) {
       uint8_t* v = smem + kOffKv + (side * kKvStages + stage) * kKvStageBytes + kKBytes;
       for (int bx = 0; bx < kBoxes; ++bx)
-        for (int idx = valid * 8 + lane; idx < BKV * 8; idx += 32)
+        for (int idx = valid * (C::kRowBytes / 16) + lane; idx < BKV * (C::kRowBytes / 16); idx += 32)
           *reinterpret_cast<uint4*>(v + bx * C::kKvBoxBytes + idx * 16) = make_uint4(0u, 0u, 0u, 0u);
       fence_proxy_async_smem();
       __syncwarp();
@@ -585,8 +596,12 @@ dca_umma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
         const float l_tot = half == 0 ? l_run + l_o : l_o + l_run;  // same order in both halves
         const float inv = 1.f / l_tot;
         uint32_t v[kOutCols];
+        if constexpr (kOutCols == 16) {
+          tmem_ld_32x32b_x16(t_o, v);
+        } else {
 #pragma unroll
-        for (int c = 0; c < kOutCols; c += 32) tmem_ld_32x32b_x32(t_o + c, v + c);
+          for (int c = 0; c < kOutCols; c += 32) tmem_ld_32x32b_x32(t_o + c, v + c);
+        }
         tmem_ld_wait();
         // Scores that outgrow the first block's maximum by 2^128 or so overflow fp32 (and so can
         // a sum of products with huge values): the row then holds Inf or NaN instead of a result.
@@ -644,7 +659,7 @@ int sm_count_dca() {
 }  // namespace
 
 bool umma_dca_supported(int32_t n_q, int32_t H, int32_t dh) {
-  return (dh == 64 || dh == 128) && n_q >= 1 && n_q <= BQ && H >= 1 && H <= 65535;
+  return (dh == 32 || dh == 64 || dh == 128) && n_q >= 1 && n_q <= BQ && H >= 1 && H <= 65535;
 }
 
 template <int DH, int BKV>
@@ -658,12 +673,15 @@ static rocs_status_t launch_dca(const rocs_plan* plan, int32_t n_q, int32_t H, f
   if (items.num == 0) return ROCS_OK;
   const uint64_t width = (uint64_t)H * DH;
   CUtensorMap map_q, map_k, map_v;
-  if (!make_tensor_map_2d(&map_q, Q, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, (uint64_t)plan->N * n_q, width, width, BQ, 64,
-                          true))
+  constexpr bool sw64 = C::kRowBytes == 64;
+  if (!make_tensor_map_2d(&map_q, Q, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, (uint64_t)plan->N * n_q, width, width, BQ,
+                          C::kBoxCols, true, sw64))
     return ROCS_ERR_CUDA;
   if (T > 0) {
-    if (!make_tensor_map_2d(&map_k, K, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, (uint64_t)T, width, width, BKV, 64, true) ||
-        !make_tensor_map_2d(&map_v, V, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, (uint64_t)T, width, width, BKV, 64, true))
+    if (!make_tensor_map_2d(&map_k, K, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, (uint64_t)T, width, width, BKV, C::kBoxCols,
+                            true, sw64) ||
+        !make_tensor_map_2d(&map_v, V, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, (uint64_t)T, width, width, BKV, C::kBoxCols,
+                            true, sw64))
       return ROCS_ERR_CUDA;
   } else {
     map_k = map_q;  // every sequence is empty: the kernel only writes zeros
@@ -699,6 +717,7 @@ rocs_status_t umma_dca(const rocs_plan* plan, int32_t n_q, int32_t H, int32_t dh
                        cudaStream_t stream) {
   if (plan->N == 0) return ROCS_OK;
   if (dh == 64) return launch_dca<64, 128>(plan, n_q, H, scale, Q, K, V, seq_offsets, T, O, stream);
+  if (dh == 32) return launch_dca<32, 128>(plan, n_q, H, scale, Q, K, V, seq_offsets, T, O, stream);
   return launch_dca<128, 64>(plan, n_q, H, scale, Q, K, V, seq_offsets, T, O, stream);
 }
 

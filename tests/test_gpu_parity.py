@@ -243,20 +243,23 @@ def test_dca_bf16_other_head_dims(dh):
     assert _run_dca(cfg, co, so) <= tol_for("bf16")
 
 
-def test_dca_bf16_head_dim_128_ragged_on_tensor_cores():
-    # dh = 128 runs on the tensor-core kernel with 64-key blocks: segments around the 128-row tile, empty
-    # request / sequence, lengths around the key block, several query tokens
+@pytest.mark.parametrize("dh", [32, 128])
+def test_dca_bf16_head_dim_32_and_128_ragged_on_tensor_cores(dh):
+    # dh = 128 runs on the tensor-core kernel with 64-key blocks, dh = 32 with 64-byte operand rows:
+    # segments around the 128-row tile, empty request / sequence, lengths around the key block, several
+    # query tokens
     co = wl.offsets_from_counts([1, 130, 0, 128, 17, 255])
     so = wl.offsets_from_counts([5, 128, 64, 129, 0, 300])
-    cfg = wl.CONFIGS[3].with_(R=6, H=2, dh=128)
+    cfg = wl.CONFIGS[3].with_(R=6, H=2, dh=dh)
     assert _run_dca(cfg, co, so) <= tol_for("bf16")
-    cfg = wl.CONFIGS[3].with_(R=3, H=3, dh=128, n_q=5)
+    cfg = wl.CONFIGS[3].with_(R=3, H=3, dh=dh, n_q=5)
     assert _run_dca(cfg, wl.offsets_from_counts([3, 50, 9]), wl.offsets_from_counts([70, 33, 257]), scale=0.1) <= tol_for("bf16")
 
 
-def test_dca_bf16_head_dim_128_many_tiles_sampled():
-    # enough tiles that every SM runs several items on both of its streams (L = 700: 11 key blocks)
-    cfg = wl.CONFIGS[3].with_(R=48, H=4, dh=128, L_const=700)
+@pytest.mark.parametrize("dh", [32, 128])
+def test_dca_bf16_head_dim_32_and_128_many_tiles_sampled(dh):
+    # enough tiles that every SM runs several items on both of its streams (L = 700: 11 or 6 key blocks)
+    cfg = wl.CONFIGS[3].with_(R=48, H=4, dh=dh, L_const=700)
     co, so = wl.cand_offsets(cfg), wl.seq_offsets(cfg)
     sample = wl.stratified_sample(co, n_uniform=128, n_small_requests=2, cfg_id=3)
     assert _run_dca(cfg, co, so, sample=sample) <= tol_for("bf16")
