@@ -47,7 +47,7 @@ N_SETS = 4  # rotating input/output sets: 4 x (67 MB in + 600 MB activations) >>
 # dram__bytes_read.sum + dram__bytes_write.sum per launch, from the ncu captures summarised under
 # profiles/ (bytes; the request half of layer 1 adds 1.3 MB).  Below the algorithmic bytes where the
 # tail of the output is still in L2 when the kernel ends.
-NCU_TRAFFIC = {"L1": 278.5e6 + 1.3e6, "L2": 500.6e6, "L3": 315.0e6}
+NCU_TRAFFIC = {"L1": 278.8e6 + 1.3e6, "L2": 500.8e6, "L3": 315.5e6}
 
 
 def measured_peaks():

@@ -265,6 +265,31 @@ def test_dca_bf16_head_dim_32_and_128_many_tiles_sampled(dh):
     assert _run_dca(cfg, co, so, sample=sample) <= tol_for("bf16")
 
 
+@pytest.mark.parametrize("dh", [32, 64, 128])
+def test_dca_bf16_scores_that_outgrow_the_first_key_block(dh):
+    # The tensor-core kernel fixes a row's softmax reference from its first key block.  Keys far
+    # down the sequence that are large multiples of a query row push that row's (and, through
+    # chance alignment, other rows') scores hundreds of nats above the reference, beyond what
+    # fp32 exponentials can hold: such rows must come out of the kernel's plain-fp32 recomputation,
+    # and every other row must be untouched by it.
+    co = wl.offsets_from_counts([200, 100])
+    so = wl.offsets_from_counts([600, 300])
+    cfg = wl.CONFIGS[5].with_(R=2, dh=dh)
+    d = wl.dca_inputs(cfg, co, so)
+    Q, K = wl.bf16_bits_to_f32(d["Q"]), wl.bf16_bits_to_f32(d["K"])
+    K[300] = Q[5, 0] * 60.0      # request 0, third key block: +60 |q|^2 for query row 5
+    K[450] = Q[140, 0] * 3.0
+    K[258] = Q[7, 0] * 60.0
+    K[130] = Q[150, 0] * -80.0   # second key block: huge negative for row 150, +-hundreds for the rest
+    K[700] = Q[250, 0] * 40.0    # request 1, second key block
+    d["K"] = wl.f32_to_bf16_bits(K)
+    plan = _plan(co)
+    O = rocs.dca_attention(plan, to_dev(d["Q"]), to_dev(d["K"]), to_dev(d["V"]), to_dev(so))
+    want = ref.dca_attention(co, so, d["Q"], d["K"], d["V"])
+    assert rel_err(to_host_f64(O), want) <= tol_for("bf16")
+    assert rocs.last_device_status() == 0
+
+
 def test_dca_bf16_64_query_tokens_per_candidate():
     # two candidates fill a 128-row tile (Section 4.3.2 names query tiles of 32 and 64 tokens)
     co = wl.offsets_from_counts([5, 1, 12, 2])
