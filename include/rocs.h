@@ -175,6 +175,9 @@ rocs_status_t rocs_linear(rocs_dtype_t dtype, int64_t M, int32_t d_in, int32_t d
  *   seq_offsets  [R+1] device int32, non-decreasing, [0] = 0 (contents are not validated)
  *   scale <= 0 selects 1/sqrt(dh)
  *   dh * sizeof(element) must be a multiple of 16; dh <= 256
+ * bf16 with dh in {32, 64, 128} and n_q <= 128 runs on the tensor cores; anything else on a
+ * general kernel.  Values of one request never reach another request's rows, NaN and Inf
+ * included (the invariant of Eq. 1): a NaN in K or V of request r shows in rows of r only.
  * A request with L_r = 0 yields zero rows.  `workspace` may be NULL when
  * rocs_dca_attention_workspace returns 0.
  * Errors: INVALID_ARG, ALIGNMENT, WORKSPACE, UNSUPPORTED, CUDA.

@@ -19,6 +19,7 @@
 #include <algorithm>
 
 #include "rocs_internal.h"
+#include "simt_util.cuh"
 #include "sm100_ptx.cuh"
 
 namespace rocs {
@@ -48,23 +49,42 @@ __global__ void __launch_bounds__(256) fm_request_kernel(int32_t n_r, int32_t d,
   // the candidate kernel may start now: it streams X^C on its own and waits for this grid only
   // before it reads TT
   ptx::griddep_launch_dependents();
-  for (int e = threadIdx.x; e < n_r * d; e += blockDim.x) xr[(e / d) * ds + e % d] = ld_f(XR, (int64_t)r * n_r * d + e);
+  rows_to_shared(XR + (int64_t)r * n_r * d, xr, n_r, d, ds);
   for (int e = threadIdx.x; e < n_r * k; e += blockDim.x) pr[e] = ld_f(P, e);
   __syncthreads();
-  for (int idx = threadIdx.x; idx < k * d; idx += blockDim.x) {
-    const int c = idx / d, e = idx % d;
-    float acc = 0.f;
-    for (int a = 0; a < n_r; ++a) acc = fmaf(pr[a * k + c], xr[a * ds + e], acc);
-    tt[c * ds + e] = acc;
-    TT[((int64_t)r * k + c) * d + e] = acc;
+  // TT: one column e and up to eight projection columns c per work item, i.e. eight independent sums
+  // per thread fed by one read of X^R per step
+  constexpr int kCg = 8;
+  const int n_cg = (k + kCg - 1) / kCg;
+  for (int idx = threadIdx.x; idx < n_cg * d; idx += blockDim.x) {
+    const int c0 = (idx / d) * kCg, e = idx % d;
+    float acc[kCg];
+#pragma unroll
+    for (int u = 0; u < kCg; ++u) acc[u] = 0.f;
+    for (int a = 0; a < n_r; ++a) {
+      const float x = xr[a * ds + e];
+#pragma unroll
+      for (int u = 0; u < kCg; ++u) acc[u] = fmaf(pr[a * k + min(c0 + u, k - 1)], x, acc[u]);
+    }
+#pragma unroll
+    for (int u = 0; u < kCg; ++u)
+      if (c0 + u < k) {
+        tt[(c0 + u) * ds + e] = acc[u];
+        TT[((int64_t)r * k + c0 + u) * d + e] = acc[u];
+      }
   }
   if (!FR) return;
   __syncthreads();
   for (int idx = threadIdx.x; idx < n_r * k; idx += blockDim.x) {
     const int a = idx / k, c = idx % k;
-    float acc = 0.f;
-    for (int e = 0; e < d; ++e) acc = fmaf(xr[a * ds + e], tt[c * ds + e], acc);
-    st_f(FR, ((int64_t)r * n_r + a) * k + c, acc);
+    float acc[4] = {0.f, 0.f, 0.f, 0.f};  // four chains over d, added in a fixed order
+    int e = 0;
+    for (; e + 3 < d; e += 4) {
+#pragma unroll
+      for (int u = 0; u < 4; ++u) acc[u] = fmaf(xr[a * ds + e + u], tt[c * ds + e + u], acc[u]);
+    }
+    for (; e < d; ++e) acc[0] = fmaf(xr[a * ds + e], tt[c * ds + e], acc[0]);
+    st_f(FR, ((int64_t)r * n_r + a) * k + c, (acc[0] + acc[1]) + (acc[2] + acc[3]));
   }
 }
 

@@ -3,6 +3,8 @@
 // Every output row is produced by a fixed instruction sequence over that row's own inputs, so
 // results are bitwise deterministic and independent of neighbouring candidates (Eq. 1).
 #include "rocs_internal.h"
+#include "simt_util.cuh"
+#include "sm100_ptx.cuh"
 
 namespace rocs {
 namespace {
@@ -175,8 +177,10 @@ __global__ void __launch_bounds__(256) glm_request_simt_kernel(
   float* g = xr + (size_t)n_r * ds;            // [n_r, n_r]
   float* w = g + (size_t)n_r * n_r;            // [n_ro + n_co, n_r]: the request columns of W
   const int32_t r = blockIdx.x;
-  for (int e = threadIdx.x; e < n_r * d; e += blockDim.x)
-    xr[(e / d) * ds + e % d] = ld_f(XR, (int64_t)r * n_r * d + e);
+  // a candidate kernel launched behind this one as a programmatic dependent may start now: it streams
+  // its own operands and waits for this grid only before it reads ZR
+  ptx::griddep_launch_dependents();
+  rows_to_shared(XR + (int64_t)r * n_r * d, xr, n_r, d, ds);
   if (W)
     for (int e = threadIdx.x; e < (n_ro + n_co) * n_r; e += blockDim.x)
       w[e] = ld_f(W, (int64_t)(e / n_r) * n + e % n_r);
@@ -210,8 +214,16 @@ __global__ void __launch_bounds__(256) glm_request_simt_kernel(
     for (int idx = threadIdx.x; idx < (n_ro + n_co) * n; idx += blockDim.x) {
       const int o = idx / n, b = idx % n;
       float acc = 0.f;
-      if (b < n_r)
-        for (int a = 0; a < n_r; ++a) acc = fmaf(w[o * n_r + a], g[a * n_r + b], acc);
+      if (b < n_r) {
+        float acc1 = 0.f;  // two chains: the sum is short but each step waits for two shared-memory reads
+        int a = 0;
+        for (; a + 1 < n_r; a += 2) {
+          acc = fmaf(w[o * n_r + a], g[a * n_r + b], acc);
+          acc1 = fmaf(w[o * n_r + a + 1], g[(a + 1) * n_r + b], acc1);
+        }
+        if (a < n_r) acc = fmaf(w[o * n_r + a], g[a * n_r + b], acc);
+        acc += acc1;
+      }
       if (o < n_ro) {
         if (OR_) st_f(OR_, ((int64_t)r * n_ro + o) * n + b, acc);
       } else if (ZR) {

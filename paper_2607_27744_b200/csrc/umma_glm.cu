@@ -41,6 +41,7 @@ struct GlmParams {
   int32_t stages, stage_bytes, group_staging_bytes, yc_stride;
   const __nv_bfloat16* W;  // [n_ro + n_co, n] or null
   const float* ZR;         // [R, n_co, n] or null
+  int32_t zr_from_previous_launch;  // launched as a programmatic dependent of the kernel that writes ZR
   __nv_bfloat16* YC;       // [N, n_c, n] or null
   __nv_bfloat16* OC;       // [N, n_co, n] or null
   uint32_t* status;
@@ -160,6 +161,7 @@ glm_umma_kernel(const __grid_constant__ CUtensorMap map_xr, const __grid_constan
     uint8_t* yc_w = staging + g * p.group_staging_bytes + q * 32 * p.yc_stride;
     uint8_t* my = yc_w + lane * p.yc_stride;
     const bool compress = p.W != nullptr && p.OC != nullptr;
+    bool zr_ready = !p.zr_from_previous_launch;
     // A fragments of W_CC for mma.m16n8k16 (rows = outputs o, padded to 16; cols = a, padded to
     // 16 per K step): a0 = (g8, 2t..), a1 = (g8+8, 2t..), a2 = (g8, 2t+8..), a3 = (g8+8, 2t+8..)
     constexpr int KS = (NC + 15) / 16;
@@ -246,6 +248,10 @@ glm_umma_kernel(const __grid_constant__ CUtensorMap map_xr, const __grid_constan
         // OC[c] (n_co x n) = ZR[r] + W_CC (n_co x NC) * YC[c] (NC x n) per candidate, on the warp-level
         // tensor-core path (mma.sync m16n8k16): the product is tiny and needs no TMEM round trip.
         const float* zr = p.ZR + (int64_t)tile.req * p.n_co * n;
+        if (!zr_ready) {  // the request kernel must have finished before its result is read
+          griddep_wait();
+          zr_ready = true;
+        }
         const int32_t cands = rows_valid / NC;
         for (int32_t cl = 0; cl < cands; ++cl) {
           __nv_bfloat16* oc = p.OC + ((int64_t)tile.cand0 + q * (32 / NC) + cl) * p.n_co * n;
@@ -382,11 +388,24 @@ rocs_status_t umma_glm(const rocs_plan* plan, int32_t n_r, int32_t n_c, int32_t 
   p.YC = (__nv_bfloat16*)YC; p.OC = (__nv_bfloat16*)OC;
   p.status = status;
   const int grid = std::min(tl.num, sm_count_glm());
+  // The request kernel runs directly in front on the same stream and releases its dependents at once:
+  // this kernel sets itself up and streams X^C beside it and waits for it only before it reads ZR.
+  p.zr_from_previous_launch = (zr_workspace != nullptr && W != nullptr && OC != nullptr) ? 1 : 0;
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(grid);
+  cfg.blockDim = dim3(kThreads);
+  cfg.dynamicSmemBytes = L.smem_bytes;
+  cfg.stream = stream;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = p.zr_from_previous_launch ? 1 : 0;
 #define ROCS_GLM_LAUNCH(NC_)                                                                                  \
   do {                                                                                                        \
     ROCS_CUDA_TRY(cudaFuncSetAttribute(glm_umma_kernel<NC_>, cudaFuncAttributeMaxDynamicSharedMemorySize,     \
                                        L.smem_bytes));                                                        \
-    glm_umma_kernel<NC_><<<grid, kThreads, L.smem_bytes, stream>>>(map_xr, map_xc, p);                        \
+    ROCS_CUDA_TRY(cudaLaunchKernelEx(&cfg, glm_umma_kernel<NC_>, map_xr, map_xc, p));                         \
   } while (0)
   if (n_c == 8) ROCS_GLM_LAUNCH(8);
   else if (n_c == 16) ROCS_GLM_LAUNCH(16);
