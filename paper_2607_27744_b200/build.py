@@ -10,7 +10,7 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 OBJ = os.path.join(HERE, "build")
 LIB = os.path.join(HERE, "librocs.so")
-SOURCES = ["api.cu", "simt_kernels.cu", "tensor_map.cu", "umma_linear.cu", "umma_linear_ws2.cu", "umma_linear_pair.cu", "umma_dca.cu", "umma_glm.cu", "fm_projection.cu", "group_norm.cu", "no_alloc.cu", "selftest.cu", "row_stats.cu"]
+SOURCES = ["api.cu", "simt_kernels.cu", "tensor_map.cu", "umma_linear.cu", "umma_linear_ws2.cu", "umma_linear_pair.cu", "umma_dca.cu", "umma_glm.cu", "fm_projection.cu", "group_norm.cu", "no_alloc.cu", "selftest.cu", "row_stats.cu", "glm_request_mma.cu"]
 NVCC_FLAGS = [
     "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
     "-Xcompiler", "-fPIC", "--expt-relaxed-constexpr",

@@ -486,9 +486,11 @@ rocs_status_t rocs_glm_interaction(const rocs_plan_t* plan, rocs_dtype_t dtype, 
     zr = (float*)workspace;
   }
   if (dtype == ROCS_BF16 && g_path.load() == ROCS_PATH_AUTO && umma_glm_supported(n_r, n_c, d, n_ro, n_co)) {
-    // Request side once per request on the general kernel (tiny), candidate side on tensor cores.
-    rocs_status_t st = simt_glm(dtype, plan, n_r, n_c, d, XR, nullptr, W, n_ro, n_co, YR, nullptr, OR_,
-                                nullptr, zr, stream);
+    // Request side once per request (tiny), candidate side on tensor cores.
+    rocs_status_t st = glm_request_mma_supported(n_r, d, n_ro, n_co)
+                           ? glm_request_mma(plan, n_r, n_c, d, XR, W, n_ro, n_co, YR, OR_, zr, stream)
+                           : simt_glm(dtype, plan, n_r, n_c, d, XR, nullptr, W, n_ro, n_co, YR, nullptr, OR_,
+                                      nullptr, zr, stream);
     if (st != ROCS_OK) return st;
     if (!YC && !OC) return ROCS_OK;
     return umma_glm(plan, n_r, n_c, d, XR, XC, W, n_ro, n_co, YC, OC, zr, stream);

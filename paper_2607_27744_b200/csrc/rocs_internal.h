@@ -156,6 +156,13 @@ rocs_status_t umma_glm(const rocs_plan* plan, int32_t n_r, int32_t n_c, int32_t 
                        const void* XC, const void* W, int32_t n_ro, int32_t n_co, void* YC,
                        void* OC, const float* zr_workspace, cudaStream_t stream);
 
+// Request side of the interaction operator on warp-level tensor cores (bf16): YR, OR and the request
+// term ZR of the compression, one block per request.
+bool glm_request_mma_supported(int32_t n_r, int32_t d, int32_t n_ro, int32_t n_co);
+rocs_status_t glm_request_mma(const rocs_plan* plan, int32_t n_r, int32_t n_c, int32_t d, const void* XR,
+                              const void* W, int32_t n_ro, int32_t n_co, void* YR, void* OR_, float* zr,
+                              cudaStream_t stream);
+
 // Device status word written by bounded waits of the tensor-core kernels.
 uint32_t* device_status_word();
 
