@@ -153,6 +153,112 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
   return *reinterpret_cast<const uint32_t*>(&h);
 }
 
+// ---------------------------------------------------------------------------------------------
+// Request side on warp-level tensor cores (bf16; k and d multiples of 8 and 16): the same two products
+// as fm_request_kernel out of bf16 copies of X^R_r and P_R in shared memory.
+//   TT[c][e] = sum_a P_R[a][c] X^R[a][e]   A = P_R^T and B = X^R, both read with ldmatrix.trans
+//   FR[a][c] = sum_e X^R[a][e] TT[c][e]    A = X^R rows, B = rows of TT: TT enters as a bf16 pair
+//                                          (value rounded to bf16 + the rounded remainder), two products,
+//                                          so FR keeps fp32-level accuracy (relative error 2^-17)
+// ---------------------------------------------------------------------------------------------
+__device__ __forceinline__ void ldmatrix_x2(uint32_t addr, uint32_t (&r)[2]) {
+  asm volatile("ldmatrix.sync.aligned.m8n8.x2.shared.b16 {%0, %1}, [%2];" : "=r"(r[0]), "=r"(r[1]) : "r"(addr));
+}
+
+__global__ void __launch_bounds__(256) fm_request_mma_kernel(int32_t n_r, int32_t d, int32_t k,
+                                                             const __nv_bfloat16* __restrict__ XR,
+                                                             const __nv_bfloat16* __restrict__ P, float* __restrict__ TT,
+                                                             __nv_bfloat16* __restrict__ FR) {
+  extern __shared__ __align__(16) uint8_t smem_fmr[];
+  const int32_t n_rp = (n_r + 15) / 16 * 16, kp = (k + 15) / 16 * 16;
+  const int32_t x_row = (d + 8) * 2, p_row = (kp + 8) * 2;  // bytes; 16 mod 32: ldmatrix without bank conflicts
+  uint8_t* xb = smem_fmr;                    // [n_rp][d + 8] bf16, padding rows zero
+  uint8_t* pb = xb + (size_t)n_rp * x_row;   // [n_rp][kp + 8] bf16, padding rows and columns zero
+  uint8_t* th = pb + (size_t)n_rp * p_row;   // [kp][d + 8] bf16: TT rounded
+  uint8_t* tl = th + (size_t)kp * x_row;     // [kp][d + 8] bf16: what the rounding left
+  const int32_t r = blockIdx.x;
+  const int warp = threadIdx.x / 32, lane = threadIdx.x % 32;
+  ptx::griddep_launch_dependents();
+
+  const int32_t vpr = d / 8, n_vec = n_r * vpr;
+  const uint4* src = reinterpret_cast<const uint4*>(XR + (int64_t)r * n_r * d);
+  for (int32_t base = threadIdx.x; base < n_vec; base += 4 * 256) {
+    uint4 raw[4];
+#pragma unroll
+    for (int u = 0; u < 4; ++u)
+      if (base + u * 256 < n_vec) raw[u] = __ldg(src + base + u * 256);
+#pragma unroll
+    for (int u = 0; u < 4; ++u) {
+      const int32_t v = base + u * 256;
+      if (v < n_vec) *reinterpret_cast<uint4*>(xb + (v / vpr) * x_row + (v % vpr) * 16) = raw[u];
+    }
+  }
+  for (int32_t v = n_vec + threadIdx.x; v < n_rp * vpr; v += 256)
+    *reinterpret_cast<uint4*>(xb + (v / vpr) * x_row + (v % vpr) * 16) = make_uint4(0u, 0u, 0u, 0u);
+  for (int32_t e = threadIdx.x; e < n_rp * kp; e += 256) {
+    const int32_t a = e / kp, c = e % kp;
+    reinterpret_cast<__nv_bfloat16*>(pb + a * p_row)[c] = (a < n_r && c < k) ? P[a * k + c] : __float2bfloat16_rn(0.f);
+  }
+  __syncthreads();
+
+  const uint32_t xb_a = smem_u32(xb), pb_a = smem_u32(pb), th_a = smem_u32(th), tl_a = smem_u32(tl);
+  const int g8 = lane / 4, t4 = lane % 4;
+  const int lr = lane & 7, lq = lane >> 3;  // row inside an 8x8 block, which of the four blocks
+  // ---- TT: 16 projection columns (one M tile per 16 of kp) x pairs of 8-wide column tiles of d
+  const int32_t n_pairs = d / 16;
+  for (int32_t t = warp; t < (kp / 16) * n_pairs; t += 8) {
+    const int32_t c0 = (t / n_pairs) * 16, e0 = (t % n_pairs) * 16;
+    float acc[2][4] = {{0.f, 0.f, 0.f, 0.f}, {0.f, 0.f, 0.f, 0.f}};
+    for (int32_t a0 = 0; a0 < n_rp; a0 += 16) {
+      uint32_t fa[4], fb[4];
+      // A = P_R^T: blocks (c lo, a lo), (c hi, a lo), (c lo, a hi), (c hi, a hi) of the transposed tile
+      ldmatrix_x4_trans(pb_a + (a0 + lr + (lq >> 1) * 8) * p_row + (c0 + (lq & 1) * 8) * 2, fa);
+      // B = X^R: blocks (a lo, e lo), (a hi, e lo), (a lo, e hi), (a hi, e hi)
+      ldmatrix_x4_trans(xb_a + (a0 + lr + (lq & 1) * 8) * x_row + (e0 + (lq >> 1) * 8) * 2, fb);
+      mma_bf16(acc[0], fa, fb[0], fb[1]);
+      mma_bf16(acc[1], fa, fb[2], fb[3]);
+    }
+#pragma unroll
+    for (int h = 0; h < 2; ++h)
+#pragma unroll
+      for (int j = 0; j < 2; ++j) {
+        const int32_t c = c0 + g8 + j * 8, e = e0 + h * 8 + 2 * t4;
+        const float v0 = acc[h][2 * j], v1 = acc[h][2 * j + 1];
+        if (c < k) *reinterpret_cast<float2*>(TT + ((int64_t)r * k + c) * d + e) = make_float2(v0, v1);
+        const __nv_bfloat162 hi = __floats2bfloat162_rn(v0, v1);
+        const __nv_bfloat162 lo = __floats2bfloat162_rn(v0 - __low2float(hi), v1 - __high2float(hi));
+        *reinterpret_cast<__nv_bfloat162*>(th + c * x_row + e * 2) = hi;
+        *reinterpret_cast<__nv_bfloat162*>(tl + c * x_row + e * 2) = lo;
+      }
+  }
+  if (!FR) return;
+  __syncthreads();
+  // ---- FR: 16 x 8 tiles over (a, c)
+  const int32_t n_ct = kp / 8;
+  for (int32_t t = warp; t < (n_rp / 16) * n_ct; t += 8) {
+    const int32_t a0 = (t / n_ct) * 16, c0 = (t % n_ct) * 8;
+    const uint32_t a_addr = xb_a + (a0 + lr + (lq & 1) * 8) * x_row + (lq >> 1) * 16;
+    const uint32_t b_off = (c0 + lr) * x_row + (lq & 1) * 16;
+    float acc[4] = {0.f, 0.f, 0.f, 0.f};
+    for (int32_t e0 = 0; e0 < d; e0 += 16) {
+      uint32_t fa[4], bh[2], bl[2];
+      ldmatrix_x4(a_addr + e0 * 2, fa);
+      ldmatrix_x2(th_a + b_off + e0 * 2, bh);
+      ldmatrix_x2(tl_a + b_off + e0 * 2, bl);
+      mma_bf16(acc, fa, bh[0], bh[1]);
+      mma_bf16(acc, fa, bl[0], bl[1]);
+    }
+#pragma unroll
+    for (int h = 0; h < 2; ++h) {
+      const int32_t a = a0 + g8 + h * 8, c = c0 + 2 * t4;
+      if (a < n_r) {
+        if (c < k) FR[((int64_t)r * n_r + a) * k + c] = __float2bfloat16_rn(acc[2 * h]);
+        if (c + 1 < k) FR[((int64_t)r * n_r + a) * k + c + 1] = __float2bfloat16_rn(acc[2 * h + 1]);
+      }
+    }
+  }
+}
+
 struct FmParams {
   int64_t N;
   int32_t n_r, k, num_tiles;
@@ -371,7 +477,14 @@ rocs_status_t launch_fm(const rocs_plan* plan, int32_t n_r, int32_t n_c, int32_t
   const size_t smem_r = ((size_t)(n_r + k) * (d + 1) + (size_t)n_r * k) * sizeof(float);
   const size_t smem_c = ((size_t)(n_c + k) * (d + 1) + (size_t)n_c * k) * sizeof(float);
   if (smem_r > kMaxSmem || smem_c > kMaxSmem) return ROCS_ERR_UNSUPPORTED;
-  if (plan->R > 0) {
+  const size_t n_rp = (size_t)(n_r + 15) / 16 * 16, kp = (size_t)(k + 15) / 16 * 16;
+  const size_t smem_mma = n_rp * ((size_t)(d + 8) * 2 + (kp + 8) * 2) + 2 * kp * (size_t)(d + 8) * 2;
+  if (plan->R > 0 && sizeof(T) == 2 && d % 16 == 0 && k % 8 == 0 && smem_mma <= kMaxSmem) {
+    ROCS_CUDA_TRY(cudaFuncSetAttribute(fm_request_mma_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_mma));
+    fm_request_mma_kernel<<<plan->R, 256, smem_mma, stream>>>(n_r, d, k, (const __nv_bfloat16*)XR,
+                                                              (const __nv_bfloat16*)P, TT, (__nv_bfloat16*)FR);
+    ROCS_CUDA_TRY(cudaGetLastError());
+  } else if (plan->R > 0) {
     ROCS_CUDA_TRY(cudaFuncSetAttribute(fm_request_kernel<T>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kMaxSmem));
     fm_request_kernel<T><<<plan->R, 256, smem_r, stream>>>(n_r, d, k, (const T*)XR, (const T*)P, TT, (T*)FR);
     ROCS_CUDA_TRY(cudaGetLastError());
