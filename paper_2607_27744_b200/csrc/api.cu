@@ -2,6 +2,8 @@
 #include <algorithm>
 #include <atomic>
 #include <cmath>
+#include <map>
+#include <mutex>
 #include <new>
 
 #include "rocs_internal.h"
@@ -31,6 +33,38 @@ bool row_stride_ok(int64_t ld, int64_t min_cols, rocs_dtype_t dt) {
 __device__ uint32_t g_device_status;
 
 }  // namespace
+
+// Stream-ordered allocations of the plan (request ids, work lists) come from a pool of the library's
+// own that keeps freed memory instead of returning it to the driver at the next synchronisation: a
+// serving loop builds and drops one plan per batch, and with the default pool's zero release
+// threshold every batch would pay the driver's allocation path again.
+static cudaError_t pool_alloc(void** ptr, size_t bytes, cudaStream_t stream) {
+  static std::mutex mu;
+  static std::map<int, cudaMemPool_t> pools;
+  int dev = 0;
+  cudaError_t e = cudaGetDevice(&dev);
+  if (e != cudaSuccess) return e;
+  cudaMemPool_t pool = nullptr;
+  {
+    std::lock_guard<std::mutex> lock(mu);
+    auto it = pools.find(dev);
+    if (it == pools.end()) {
+      cudaMemPoolProps props = {};
+      props.allocType = cudaMemAllocationTypePinned;
+      props.handleTypes = cudaMemHandleTypeNone;
+      props.location.type = cudaMemLocationTypeDevice;
+      props.location.id = dev;
+      e = cudaMemPoolCreate(&pool, &props);
+      if (e != cudaSuccess) return e;
+      uint64_t keep = UINT64_MAX;
+      cudaMemPoolSetAttribute(pool, cudaMemPoolAttrReleaseThreshold, &keep);
+      pools[dev] = pool;
+    } else {
+      pool = it->second;
+    }
+  }
+  return cudaMallocFromPoolAsync(ptr, bytes, pool, stream);
+}
 
 uint32_t* device_status_word() {
   uint32_t* p = nullptr;
@@ -89,7 +123,7 @@ static rocs_status_t upload_entry_base(const rocs_plan* plan, int32_t per_entry,
   }
   base[plan->R] = (int32_t)acc;
   *total = acc;
-  ROCS_CUDA_TRY(cudaMallocAsync((void**)base_dev, sizeof(int32_t) * base.size(), stream));
+  ROCS_CUDA_TRY(pool_alloc((void**)base_dev, sizeof(int32_t) * base.size(), stream));
   // Pageable source: the copy is staged before the call returns, so `base` may go away.
   if (cudaMemcpyAsync(*base_dev, base.data(), sizeof(int32_t) * base.size(), cudaMemcpyHostToDevice, stream) !=
       cudaSuccess) {
@@ -115,7 +149,7 @@ rocs_status_t plan_tiles(const rocs_plan* plan, int32_t cands_per_tile, cudaStre
     rocs_status_t st = upload_entry_base(plan, cands_per_tile, stream, &base_dev, &total);
     if (st != ROCS_OK) return st;
     tl.num = (int32_t)total;
-    cudaError_t e = cudaMallocAsync((void**)&tl.dev, sizeof(Tile) * (size_t)total, stream);
+    cudaError_t e = pool_alloc((void**)&tl.dev, sizeof(Tile) * (size_t)total, stream);
     if (e == cudaSuccess) {
       expand_tiles_kernel<<<(unsigned)((total + 255) / 256), 256, 0, stream>>>(plan->R, tl.num, cands_per_tile,
                                                                               plan->cand_offsets, base_dev, tl.dev);
@@ -154,7 +188,7 @@ rocs_status_t plan_dca_items(const rocs_plan* plan, int32_t cands_per_tile, int3
       return ROCS_ERR_UNSUPPORTED;
     }
     il.num = (int32_t)total;
-    cudaError_t e = cudaMallocAsync((void**)&il.dev, sizeof(DcaItem) * (size_t)total, stream);
+    cudaError_t e = pool_alloc((void**)&il.dev, sizeof(DcaItem) * (size_t)total, stream);
     if (e == cudaSuccess) {
       expand_dca_items_kernel<<<(unsigned)((total + 255) / 256), 256, 0, stream>>>(
           plan->R, il.num, cands_per_tile, heads, tiles_per_item, plan->cand_offsets, base_dev, il.dev);
@@ -251,7 +285,7 @@ rocs_status_t rocs_plan_create(rocs_plan_t** out, int32_t R, int64_t N, const in
   if (N > 0) {
     // Stream-ordered allocation: after the first batch the pool hands the block back without a
     // device synchronisation, so building a plan per batch stays off the critical path.
-    if (cudaMallocAsync((void**)&p->row2req, sizeof(int32_t) * (size_t)N, stream) != cudaSuccess) {
+    if (pool_alloc((void**)&p->row2req, sizeof(int32_t) * (size_t)N, stream) != cudaSuccess) {
       delete p;
       return ROCS_ERR_CUDA;
     }
