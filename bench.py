@@ -450,6 +450,20 @@ def run_rocs(args):
     e2e_ms = max_over_ranks(e0.elapsed_time(e1)) / args.steps
     h2d = XR_h.numel() * 2 + XC_h.numel() * 2 + co_h.numel() * 4
     d2h = y_h[0].numel() * 2
+    # the step's copies alone, both directions at once: what the PCIe link allows for these bytes
+    def copies_only(n):
+        for i in range(n):
+            with torch.cuda.stream(s_in):
+                in_d[i % 2][1].copy_(XC_h, non_blocking=True)
+                in_d[i % 2][0].copy_(XR_h, non_blocking=True)
+            with torch.cuda.stream(s_out):
+                y_h[i % 2].copy_(y[i % N_SETS], non_blocking=True)
+    copies_only(3)
+    torch.cuda.synchronize()
+    t_c0 = time.perf_counter()
+    copies_only(20)
+    torch.cuda.synchronize()
+    copies_ms = (time.perf_counter() - t_c0) / 20 * 1e3
     del XR_sets, XC_sets, h1, h2, y, in_d, y_h, XR_h, XC_h
     torch.cuda.empty_cache()
 
@@ -498,7 +512,10 @@ def run_rocs(args):
                                f"(sharding.shard_batch), {shard.requests.size} requests / {N} candidates per rank"},
         "clocks": clock_summary,
         "e2e": {"value": world * N / (e2e_ms * 1e-3), "unit": UNIT, "h2d_bytes_per_step": h2d,
-                "d2h_bytes_per_step": d2h, "ms_per_step": e2e_ms},
+                "d2h_bytes_per_step": d2h, "ms_per_step": e2e_ms,
+                "copies_only_ms_per_step": copies_ms, "frac_of_copies_only": copies_ms / e2e_ms,
+                "note": "copies_only: the step's host-to-device and device-to-host copies alone, both directions "
+                        "at once, no kernels (host clock over 20 steps): the PCIe floor of this step"},
         "gpu_launches": launches_per_step * args.steps,
         "roofline": roofline,
         "dominant_launch": dominant,
