@@ -330,6 +330,29 @@ def run_rocs(args):
     torch.cuda.synchronize()
     warm = [span_median(warm_marks, a, a + 1) for a in (1, 2, 3)]
 
+    # The HBM roof under the same conditions: a plain device copy of one activation (read + write,
+    # larger than L2), timed (i) back to back after a pause, as the measured peak was, and (ii) between
+    # the steps of a long run, where the power cap has lowered the clocks.  Reported beside the roofline;
+    # the roofline's denominator stays the measured peak.
+    def copy_gbs(in_step, reps):
+        ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(reps)]
+        for i, (a_, b_) in enumerate(ev):
+            if in_step:
+                step(i)
+            a_.record()
+            h2[(i + 1) % N_SETS].copy_(h1[i % N_SETS])
+            b_.record()
+        torch.cuda.synchronize()
+        t_ = float(np.median([a_.elapsed_time(b_) for a_, b_ in ev])) * 1e-3
+        return 2.0 * h1[0].numel() * 2 / t_ / 1e9
+    time.sleep(0.5)
+    copy_alone = copy_gbs(False, 10)
+    copy_in_step = copy_gbs(True, min(args.steps, 400))
+    hbm_copy = {"alone_gbs": copy_alone, "between_steps_gbs": copy_in_step, "bytes": 2 * h1[0].numel() * 2,
+
+                "note": "torch copy_ of one 131072 x 1024 bf16 activation (read + write); between_steps: median over "
+                        "copies placed between the steps of a run of up to 400 steps"}
+
     def time_call(fn, reps=20, warm=3):
         for i in range(warm):
             fn(i)
@@ -519,6 +542,7 @@ def run_rocs(args):
         "gpu_launches": launches_per_step * args.steps,
         "roofline": roofline,
         "dominant_launch": dominant,
+        "hbm_copy": hbm_copy,
         "cpu_baseline": cpu,
         "layers": layers,
         "plan_us": t_plan * 1e6, "plan_us_in_step": t_plan_in * 1e6,
