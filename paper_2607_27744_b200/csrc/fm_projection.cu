@@ -472,14 +472,14 @@ rocs_status_t launch_fm_mma(const rocs_plan* plan, int32_t n_r, int32_t k, const
 template <typename T>
 rocs_status_t launch_fm(const rocs_plan* plan, int32_t n_r, int32_t n_c, int32_t d, int32_t k, const void* XR,
                         const void* XC, const void* P, void* FR, void* FC, float* TT, bool fast_candidates,
-                        cudaStream_t stream) {
+                        bool tensor_core_request, cudaStream_t stream) {
   constexpr size_t kMaxSmem = 200 * 1024;
   const size_t smem_r = ((size_t)(n_r + k) * (d + 1) + (size_t)n_r * k) * sizeof(float);
   const size_t smem_c = ((size_t)(n_c + k) * (d + 1) + (size_t)n_c * k) * sizeof(float);
   if (smem_r > kMaxSmem || smem_c > kMaxSmem) return ROCS_ERR_UNSUPPORTED;
   const size_t n_rp = (size_t)(n_r + 15) / 16 * 16, kp = (size_t)(k + 15) / 16 * 16;
   const size_t smem_mma = n_rp * ((size_t)(d + 8) * 2 + (kp + 8) * 2) + 2 * kp * (size_t)(d + 8) * 2;
-  if (plan->R > 0 && sizeof(T) == 2 && d % 16 == 0 && k % 8 == 0 && smem_mma <= kMaxSmem) {
+  if (plan->R > 0 && tensor_core_request && sizeof(T) == 2 && d % 16 == 0 && k % 8 == 0 && smem_mma <= kMaxSmem) {
     ROCS_CUDA_TRY(cudaFuncSetAttribute(fm_request_mma_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_mma));
     fm_request_mma_kernel<<<plan->R, 256, smem_mma, stream>>>(n_r, d, k, (const __nv_bfloat16*)XR,
                                                               (const __nv_bfloat16*)P, TT, (__nv_bfloat16*)FR);
@@ -516,9 +516,9 @@ rocs_status_t fm_projection(rocs_dtype_t dt, const rocs_plan* plan, int32_t n_r,
                             const void* XR, const void* XC, const void* P, void* FR, void* FC, float* tt_workspace,
                             bool allow_fast, cudaStream_t stream) {
   if (dt == ROCS_F32)
-    return launch_fm<float>(plan, n_r, n_c, d, k, XR, XC, P, FR, FC, tt_workspace, false, stream);
+    return launch_fm<float>(plan, n_r, n_c, d, k, XR, XC, P, FR, FC, tt_workspace, false, false, stream);
   return launch_fm<__nv_bfloat16>(plan, n_r, n_c, d, k, XR, XC, P, FR, FC, tt_workspace,
-                                  allow_fast && fm_projection_fast_supported(n_c, d, k), stream);
+                                  allow_fast && fm_projection_fast_supported(n_c, d, k), allow_fast, stream);
 }
 
 }  // namespace rocs
