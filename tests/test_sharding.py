@@ -54,7 +54,30 @@ def test_replicated_global_batch_shards_into_equal_weak_scaling_pieces():
         assert np.array_equal(np.sort(rows), np.arange(glob[-1]))
 
 
-def _worker(rank, world, port, out_q):
+def test_oversized_request_is_cut_and_every_candidate_is_scored_once():
+    """One request with most of the batch's candidates cannot be balanced whole: with max_share its
+    candidates go to several ranks (each with a copy of the request's own tensors), every candidate row
+    is owned exactly once, and the ranks' loads are even."""
+    co = wl.offsets_from_counts([5, 4000, 0, 7, 300, 12])
+    so = wl.offsets_from_counts([40, 100, 7, 0, 64, 33])
+    for world in (2, 4):
+        whole = [sharding.shard_batch(co, world, r) for r in range(world)]
+        assert max(int(s.cand_offsets[-1]) for s in whole) >= 4000           # the request cannot be balanced whole
+        cut = [sharding.shard_batch(co, world, r, seq_offsets=so, max_share=0.5) for r in range(world)]
+        rows = np.concatenate([s.cand_rows for s in cut])
+        assert np.array_equal(np.sort(rows), np.arange(co[-1]))
+        loads = np.array([int(s.cand_offsets[-1]) for s in cut])
+        assert loads.max() - loads.min() <= 8
+        for s in cut:
+            # local offsets describe the rows, and every local request carries its own sequence
+            assert s.cand_offsets[-1] == s.cand_rows.size and s.cand_offsets.size == s.requests.size + 1
+            assert np.array_equal(np.diff(s.seq_offsets), np.diff(so)[s.requests])
+            m = np.repeat(s.requests, np.diff(s.cand_offsets))
+            assert np.array_equal(m, np.searchsorted(co, s.cand_rows, side="right") - 1)   # rows belong to their request
+        assert sum(1 for s in cut if 1 in s.requests) >= 2                   # request 1 really is on several ranks
+
+
+def _worker(rank, world, port, out_q, max_share=None):
     sys.path.insert(0, ROOT)
     from oracle import rocs_ref as ref
     os.environ["MASTER_ADDR"] = "127.0.0.1"
@@ -62,8 +85,10 @@ def _worker(rank, world, port, out_q):
     dist.init_process_group("gloo", rank=rank, world_size=world)
     cfg = wl.CONFIGS[1].with_(R=7)
     co, so = wl.cand_offsets(cfg), wl.seq_offsets(cfg)
+    if max_share is not None:   # one request dominates the batch
+        co = wl.offsets_from_counts([3, 90, 0, 5, 2, 7, 1])
     lin, att = wl.linear_inputs(cfg, co), wl.dca_inputs(cfg, co, so)
-    sh = sharding.shard_batch(co, world, rank, seq_offsets=so, c_attn=0.05)   # the helper bench.py --gpus N uses
+    sh = sharding.shard_batch(co, world, rank, seq_offsets=so, c_attn=0.05, max_share=max_share)   # the helper bench.py --gpus N uses
     mine, rows, co_l, seq_rows, so_l = sh.requests, sh.cand_rows, sh.cand_offsets, sh.seq_rows, sh.seq_offsets
     y = ref.ikbo_linear(co_l, lin["XR"][mine], lin["XC"][rows], lin["W"])
     o = ref.dca_attention(co_l, so_l, att["Q"][rows], att["K"][seq_rows], att["V"][seq_rows])
@@ -88,11 +113,12 @@ def _worker(rank, world, port, out_q):
     dist.destroy_process_group()
 
 
-def test_two_gloo_ranks_reproduce_the_unsharded_result():
+@pytest.mark.parametrize("max_share", [None, 0.5])
+def test_two_gloo_ranks_reproduce_the_unsharded_result(max_share):
     ctx = mp.get_context("spawn")
     q = ctx.Queue()
-    port = 29500 + os.getpid() % 2000
-    procs = [ctx.Process(target=_worker, args=(r, 2, port, q)) for r in range(2)]
+    port = 29500 + os.getpid() % 2000 + (0 if max_share is None else 2000)
+    procs = [ctx.Process(target=_worker, args=(r, 2, port, q, max_share)) for r in range(2)]
     for p in procs:
         p.start()
     res = q.get(timeout=180)
