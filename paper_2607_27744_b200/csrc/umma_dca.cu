@@ -125,13 +125,9 @@ struct DcaParams {
 };
 
 __device__ __forceinline__ float ex2(float x) {
-#ifdef ROCS_DCA_PROBE_NOEXP
-  return x * 0.001f;  // timing probe only: wrong results
-#else
   float y;
   asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
   return y;
-#endif
 }
 
 // Packed fp32 pairs (one instruction for two lanes of arithmetic) and the three-input maximum.
