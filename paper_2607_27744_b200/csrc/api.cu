@@ -16,6 +16,8 @@ std::atomic<int> g_path{ROCS_PATH_AUTO};
 // m_i of Section 4.1 from the segment offsets: one thread per candidate, binary search.
 __global__ void fill_row2req_kernel(int32_t R, int64_t N, const int32_t* __restrict__ off,
                                     int32_t* __restrict__ row2req) {
+  // the first layer's kernel may set itself up beside this one; it waits for this grid before it reads anything
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
   const int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
   if (i >= N) return;
   int32_t lo = 0, hi = R;  // largest r with off[r] <= i

@@ -96,8 +96,12 @@ linear_umma_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_const
   __syncthreads();
   tc_fence_after_sync();
   const uint32_t tmem_base = *tmem_ptr;
-  // A dependent kernel launched with programmatic serialization (the candidate half behind the
-  // request half) may begin its own set-up now; it waits for this grid before it reads our output.
+  // Launched as a programmatic dependent: the set-up above may overlap the end of the kernel in front;
+  // nothing below touches global memory before that kernel is complete.  Then the kernel behind this one
+  // (the candidate half behind the request half) may begin its own set-up; it waits for this grid before
+  // it reads our output, and since it is released only after the wait above, everything in front of this
+  // kernel is complete by the time it starts.
+  griddep_wait();
   griddep_launch_dependents();
 
   if (warp == 0) {
@@ -295,7 +299,17 @@ rocs_status_t launch(int64_t M, int32_t d_in, int32_t d_out, const void* X, int6
   const int64_t tiles = ((M + BM - 1) / BM) * ((d_out + BN - 1) / BN);
   const int grid = (int)std::min<int64_t>(tiles, sm_count());
   LinearParams p{M, d_in, d_out, bias, add, ld_add, row2req, act, status};
-  kernel<<<grid, kThreads, Cfg::kSmemBytes, stream>>>(map_x, map_w, map_y, p);
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(grid);
+  cfg.blockDim = dim3(kThreads);
+  cfg.dynamicSmemBytes = Cfg::kSmemBytes;
+  cfg.stream = stream;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  ROCS_CUDA_TRY(cudaLaunchKernelEx(&cfg, kernel, map_x, map_w, map_y, p));
   ROCS_CUDA_TRY(cudaGetLastError());
   return ROCS_OK;
 }

@@ -88,6 +88,12 @@ linear_pair_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_const
   cluster_sync_all();
   tc_fence_after_sync();
   const uint32_t tmem_base = *tmem_ptr;
+  // Launched as a programmatic dependent: everything above (barriers, tensor memory) may run while the
+  // kernel in front of this one on the stream finishes; nothing below touches global memory before that
+  // kernel is complete.  The next kernel on the stream is released only after this wait, so whatever
+  // it may assume about its predecessors holds transitively.
+  griddep_wait();
+  griddep_launch_dependents();
 
   if (warp == 0) {
     // ------------------------------ TMA producer (both CTAs) -------------------------------
@@ -295,8 +301,17 @@ rocs_status_t umma_linear_pair(int64_t M, int32_t d_in, int32_t d_out, const voi
   const int64_t tiles = ((M + 2 * BM - 1) / (2 * BM)) * ((d_out + BN - 1) / BN);
   const int pairs = (int)std::min<int64_t>(tiles, sm_count_pair() / 2);
   ROCS_CUDA_TRY(cudaFuncSetAttribute(linear_pair_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes));
-  linear_pair_kernel<<<2 * pairs, kThreads, kSmemBytes, stream>>>(map_x, map_w, map_y, p);
-  ROCS_CUDA_TRY(cudaGetLastError());
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(2 * pairs);
+  cfg.blockDim = dim3(kThreads);
+  cfg.dynamicSmemBytes = kSmemBytes;
+  cfg.stream = stream;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  ROCS_CUDA_TRY(cudaLaunchKernelEx(&cfg, linear_pair_kernel, map_x, map_w, map_y, p));
   return ROCS_OK;
 }
 

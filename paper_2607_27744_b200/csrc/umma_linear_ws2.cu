@@ -117,6 +117,9 @@ linear_ws2_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_consta
   cluster_sync_all();  // barriers of both CTAs are initialised before anything signals across the pair
   tc_fence_after_sync();
   const uint32_t tmem_base = *tmem_ptr;
+  // A kernel launched behind this one as a programmatic dependent (the next layer) may set itself up as
+  // SMs become free; it waits for this whole grid before it touches global memory.
+  griddep_launch_dependents();
 
   if (warp == 0) {
     // ------------------------------ TMA producer (both CTAs) -------------------------------
