@@ -273,6 +273,10 @@ dca_umma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
   __syncthreads();
   tc_fence_after_sync();
   const uint32_t tmem_base = *reinterpret_cast<const uint32_t*>(smem + kOffTmemPtr);
+  // launched as a programmatic dependent: the set-up above may overlap the end of the kernel in front;
+  // global memory is touched only from here on, and the kernel behind this one is released after the wait
+  griddep_wait();
+  griddep_launch_dependents();
   const int32_t row_width = p.H * DH;  // elements per query / key row over all heads
   // Each side is a stream of its own: items 2 b + side, 2 b + side + 2 grid, ... of CTA b.
   const int32_t item0 = 2 * (int32_t)blockIdx.x, item_step = 2 * (int32_t)gridDim.x;
@@ -703,8 +707,17 @@ static rocs_status_t launch_dca(const rocs_plan* plan, int32_t n_q, int32_t H, f
   auto kernel = dca_umma_kernel<DH, BKV>;
   ROCS_CUDA_TRY(cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, C::kSmemBytes));
   const int grid = std::min((items.num + 1) / 2, sm_count_dca());  // one CTA per SM, two item streams per CTA
-  kernel<<<grid, kThreads, C::kSmemBytes, stream>>>(map_q, map_k, map_v, p);
-  ROCS_CUDA_TRY(cudaGetLastError());
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(grid);
+  cfg.blockDim = dim3(kThreads);
+  cfg.dynamicSmemBytes = C::kSmemBytes;
+  cfg.stream = stream;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  ROCS_CUDA_TRY(cudaLaunchKernelEx(&cfg, kernel, map_q, map_k, map_v, p));
   return ROCS_OK;
 }
 
