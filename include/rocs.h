@@ -17,7 +17,10 @@
  *     rows cand_offsets[r] .. cand_offsets[r+1]-1.  This is the index map m of
  *     Section 4.1 in segment form.  Empty requests are legal.
  *   - Work is enqueued on `stream` (a cudaStream_t, NULL = default stream) and the call
- *     returns without synchronising, except where stated.
+ *     returns without synchronising, except where stated.  The tensor-core kernels are
+ *     launched as programmatic dependents of the kernel in front of them on the stream: they
+ *     may set up their own on-chip state while that kernel ends, and wait for its completion
+ *     before they read or write global memory, so the ordering a stream guarantees is kept.
  *   - Errors are return codes.  Arguments are validated before anything is enqueued: every
  *     code except ROCS_ERR_CUDA means that the call launched nothing.
  *   - dtype names the storage type of all X / W / Q / K / V / output tensors of a call.
@@ -80,7 +83,8 @@ rocs_status_t rocs_set_path(rocs_path_t path);
  *                      the offsets are copied back from the device (the call synchronises
  *                      `stream`).
  * The plan owns device arrays of O(N + number of tiles) int32, allocated and freed in stream
- * order on `stream` (cudaMallocAsync); use the plan on that stream, or order other streams
+ * order on `stream` (from a memory pool of the library's own, which keeps what a destroyed plan
+ * frees for the next plan instead of returning it to the driver); use the plan on that stream, or order other streams
  * behind it yourself.  Tile lists for a given number of rows per candidate are created on
  * first use by the attention / interaction calls (one allocation + copy) and cached.
  * Errors: INVALID_ARG, SEGMENTS, CUDA.
