@@ -424,6 +424,9 @@ def run_rocs(args):
     plan_alone.close()
     for lay, t_own in zip(layers, (t_own1, t_own2, t_own3)):
         lay["us_alone_burst"] = t_own * 1e6
+    # the IKBO layer's fraction when it is not slowed by the power cap of the long run (same bytes, same peak)
+    roofline["us_alone_burst"] = layers[0]["us_alone_burst"]
+    roofline["frac_alone_burst"] = layers[0]["algorithmic_bytes"] / t_own1 / 1e9 / peaks["hbm_gbs"]
     for lay, med, w in zip(layers, medians, warm):
         lay["us_median"] = med * 1e6            # median over the timed steps (rotating sets: cold L2)
         lay["us_warm_l2"] = w * 1e6             # median of 30 steps on one buffer set
